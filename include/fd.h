@@ -1,0 +1,190 @@
+/* fd.h -- C ABI of the B200-native FlashDiffusion hot path.
+ *
+ * The library evaluates, without ever storing the N x N kernel, the Gaussian
+ * application of Sec. 2.1-2.2 of the paper
+ *
+ *     K_ij = exp(-beta * |x_i - x_j|^2)                                  (Eq. 1)
+ *     q = K 1,  K_alpha = diag(q)^-alpha K diag(q)^-alpha,  d = K_alpha 1,
+ *     s = q^-alpha * d^-1/2,   M = diag(s) K diag(s)                     (Eq. 2)
+ *     Y = M V = diag(s) K (diag(s) V)                                    (Eq. 3)
+ *
+ * tile by tile as in Eqs. 5-6, plus the drivers that sit on it: the block
+ * Rayleigh-Ritz / Lanczos eigensolver (Sec. 2.3, first paragraph), the
+ * bandwidth flow (Eqs. 7-14) and the out-of-sample extension used by the
+ * (n, beta) ladder (Sec. 1).
+ *
+ * Conventions
+ * -----------
+ * Pointers: a name ending in _dev is DEVICE memory of the GPU that was current
+ *   at fd_create; _host is host memory.  The library never allocates device
+ *   memory: every device buffer, including the workspace, is allocated and
+ *   freed by the caller and only borrowed for the duration of a call.  The
+ *   library owns the fd_ctx host object alone.
+ * Points:  X is row-major N x D float32 with row pitch ldx (elements).
+ * Blocks:  V, Y, Q0 and eigenvector outputs are COLUMN-major float32,
+ *   element (i, c) at [i + c * ld], ld >= number of rows.
+ * Streams: all work is enqueued on the cudaStream_t given at fd_create (passed
+ *   as void*; NULL = the legacy default stream).  fd_apply and fd_apply_general
+ *   return without synchronising; calls that return host scalars synchronise
+ *   that stream.
+ * Errors:  every entry point returns an fd_status; argument errors are found
+ *   before any launch; nothing aborts or throws.  There is no CPU fallback.
+ * Threads: a context is not thread-safe.
+ * k:       counts NONTRIVIAL eigenpairs; the Perron pair (eigenvalue 1) is
+ *   returned in slot 0, so k + 1 pairs come back (Sec. 2.3, Sec. 3).
+ */
+#ifndef FD_H_
+#define FD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fd_ctx fd_ctx;
+
+typedef enum {
+    FD_OK = 0,
+    FD_ERR_INVALID = 1,        /* bad argument (null, range, alignment, ld)                    */
+    FD_ERR_WORKSPACE = 2,      /* workspace too small / feature not provisioned at fd_create   */
+    FD_ERR_CUDA = 3,           /* a CUDA runtime call failed; see fd_last_error                */
+    FD_ERR_NOT_CONVERGED = 4,  /* fd_eigs hit max_applies; outputs hold the best Ritz pairs    */
+    FD_ERR_PERRON_WALL = 5,    /* Eq. 12 failed: g_P <= kappa_P * eta                          */
+    FD_ERR_UNSUPPORTED = 6,    /* shape outside what the kernels cover                         */
+    FD_ERR_TIMEOUT = 7,        /* a bounded device-side wait expired (status word set)         */
+    FD_ERR_NONFINITE = 8       /* non-finite input or intermediate detected                    */
+} fd_status;
+
+typedef enum {
+    FD_PREC_FP32 = 0,          /* fp32-grade result (relative Frobenius error <= 1e-5)         */
+    FD_PREC_FAST = 1           /* single 16-bit operands for K and V (<= 3e-3)                 */
+} fd_precision;
+
+/* Which kernel family serves the quadratic passes (fd_set_option "path"). */
+enum { FD_PATH_AUTO = 0, FD_PATH_SIMT = 1, FD_PATH_TC = 2 };
+
+/* Bytes of device workspace fd_create needs.  O(N (D + b_max + m_max)); no N^2 term.
+ * b_max: widest block passed to fd_apply / fd_apply_general (1..256).
+ * m_max: basis capacity for fd_eigs (columns); 0 if fd_eigs will not be called. */
+size_t fd_workspace_bytes(int64_t N, int32_t D, int32_t b_max, int32_t m_max);
+
+/* Creates a context over N points.  Copies X into the library's padded layouts inside the
+ * workspace (so X_dev may be released after the call), computes the column means and, if
+ * center != 0, the centred copy used by the Gram-form kernels (Eq. 4) and by fd_beta0.
+ * ws_dev must be 256-byte aligned and stay valid until fd_destroy.  Synchronises once. */
+fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int64_t ldx,
+                    int32_t center, int32_t b_max, int32_t m_max,
+                    void* ws_dev, size_t ws_bytes, void* cuda_stream);
+fd_status fd_destroy(fd_ctx* ctx);
+
+/* Tuning / test knobs by name: "path" (FD_PATH_*), "splits" (0 = auto), "flush" (column tiles
+ * between accumulator flushes of the tensor-core kernel), "poly_exp" (share of exponentials sent
+ * to the FMA pipe, 0..1).  Unknown name -> FD_ERR_INVALID. */
+fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
+fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);
+
+/* Eq. 7: beta0 = min(0.1, 1 / (2 * mean_i |x_i - mu|^2)). */
+fd_status fd_beta0(fd_ctx* ctx, double* beta0_host);
+
+/* Degree passes at bandwidth beta (Sec. 2.1 "entry fee"): q = K 1 and, for alpha != 0,
+ * d = q^-alpha * K q^-alpha; then s = q^-alpha * d^-1/2 (alpha = 0: d = q).  Sets the
+ * context's current (beta, alpha, q, d, s), which fd_apply and fd_eigs use afterwards.
+ * q_dev, d_dev, s_dev: N floats each, any may be NULL.  S_off_host receives
+ * sum_{i != j} K_ij and S_off_2beta_host the same sum for the kernel at 2 beta (obtained in
+ * the same pass from sum K_ij^2, Sec. 2.3); either may be NULL.  Synchronises. */
+fd_status fd_degree(fd_ctx* ctx, double beta, double alpha, fd_precision prec,
+                    float* q_dev, float* d_dev, float* s_dev,
+                    double* S_off_host, double* S_off_2beta_host);
+
+/* Eq. 3: Y = diag(s) K diag(s) V with the context's current beta and s.  b in 1..b_max.
+ * V_dev and Y_dev must not overlap.  Asynchronous. */
+fd_status fd_apply(fd_ctx* ctx, const float* V_dev, int64_t ldv, int32_t b,
+                   float* Y_dev, int64_t ldy, fd_precision prec);
+
+/* The single primitive of Sec. 2.1 with both diagonal scalings explicit:
+ *   Y = diag(left) K(Xrow, X) diag(right) V,  K_ij = exp(-beta |xrow_i - x_j|^2).
+ * left_dev (Nrow floats) and right_dev (N floats) may be NULL (= ones); V_dev may be NULL
+ * (= the ones vector, b must be 1).  Xrow_dev NULL means the context's own points
+ * (Nrow = N); otherwise row-major Nrow x D with pitch ldxrow, in the same coordinates as the
+ * X given to fd_create (this is the rectangular product the out-of-sample extension needs).
+ * Does not change the context's current beta.  Asynchronous. */
+fd_status fd_apply_general(fd_ctx* ctx, double beta, const float* left_dev, const float* right_dev,
+                           const float* Xrow_dev, int64_t Nrow, int64_t ldxrow,
+                           const float* V_dev, int64_t ldv, int32_t b,
+                           float* Y_dev, int64_t ldy, fd_precision prec);
+
+typedef struct {
+    int32_t applies;           /* block applications of M performed                          */
+    int32_t restarts;          /* thick restarts                                              */
+    int32_t converged;         /* leading pairs (of k + 1) with residual <= tol * theta_0     */
+    int32_t basis_cols;        /* columns in the basis at exit                                */
+    double  max_residual;      /* largest residual norm among the k + 1 returned pairs       */
+    double  seconds_apply;     /* host wall time spent inside the quadratic applies          */
+    double  seconds_total;
+} fd_eigs_info;
+
+/* Leading k + 1 eigenpairs of M = diag(s) K diag(s) at the context's current (beta, s) by block
+ * Krylov / Rayleigh-Ritz with residual expansion and thick restart (the paper names block
+ * implicitly restarted Lanczos and gives no further detail; Sec. 2.3).  b = block size,
+ * tol = residual tolerance relative to theta_0, Q0_dev = optional warm-start basis (N x q0_cols,
+ * need not be orthonormal).  evals_host: k + 1 doubles, descending.  evecs_dev: N x (k + 1)
+ * column-major, orthonormal.  Needs m_max >= 2 (k + 1) + b at fd_create.  Synchronous. */
+fd_status fd_eigs(fd_ctx* ctx, int32_t k, int32_t b, double tol, int32_t max_applies,
+                  const float* Q0_dev, int64_t ldq0, int32_t q0_cols,
+                  double* evals_host, float* evecs_dev, int64_t ldv, fd_eigs_info* info);
+
+/* One record per probe of the bandwidth flow (Eqs. 8-14). */
+typedef struct {
+    double beta, S_off, S_off_2beta, n_eff, d_hat, V_bias, V_stat, V_mach, V, g_P;
+    double lambda1;            /* first nontrivial eigenvalue                                 */
+    int32_t applies;           /* block applies the probe's eigensolve took                   */
+    int32_t flags;             /* bit 0: inadmissible (Eq. 12); bit 1: final (vertex) probe   */
+} fd_probe;
+
+typedef struct {
+    double beta_start;         /* <= 0: use Eq. 7                                             */
+    double beta_max;           /* grid end (inclusive)                                        */
+    double ratio;              /* 2 (dyadic)                                                  */
+    double alpha;
+    double eta;                /* precision scale of Eq. 11; <= 0: 1e-7 (fp32)                */
+    double tol;                /* eigensolver tolerance                                       */
+    int32_t k, b, max_applies;
+    int32_t warm_start;        /* 1: start each probe from the previous probe's eigenvectors  */
+} fd_flow_opts;
+
+enum { FD_FLOW_VERTEX = 0, FD_FLOW_PERRON_WALL = 1, FD_FLOW_LEFT_EDGE = 2, FD_FLOW_RIGHT_EDGE = 3 };
+
+/* Dyadic bandwidth flow of Sec. 2.3: probes beta_start * ratio^j, potential of Eq. 13, bracket
+ * rule and quadratic vertex, Perron wall of Eq. 12.  On return the context's current beta is
+ * beta_x and evals/evecs hold that probe's pairs.  log: capacity *n_probes records in, number
+ * written out.  Q0_dev: optional warm start for the first probe.  Synchronous. */
+fd_status fd_beta_flow(fd_ctx* ctx, const fd_flow_opts* opts, const float* Q0_dev, int64_t ldq0,
+                       int32_t q0_cols, fd_probe* log, int32_t* n_probes, int32_t* outcome,
+                       double* beta_x_host, double* evals_host, float* evecs_dev, int64_t ldv);
+
+/* Out-of-sample extension of Markov eigenvectors from the context's points to new points
+ * (Sec. 1, the (n, beta) ladder): psi_j(x) = sum_i K(x, x_i) q_i^-alpha psi_j(x_i) /
+ * (lambda_j sum_i K(x, x_i) q_i^-alpha), at the context's current (beta, alpha, q).
+ * psi_dev: N x m column-major (Markov vectors d^-1/2 * v); lambda_host: m values;
+ * out_dev: Nnew x m column-major.  Needs b_max >= m + 1.  Synchronous. */
+fd_status fd_nystrom(fd_ctx* ctx, const float* Xnew_dev, int64_t Nnew, int64_t ldxnew,
+                     const float* psi_dev, int64_t ldpsi, int32_t m, const double* lambda_host,
+                     float* out_dev, int64_t ldout);
+
+/* Elementwise helper for the end of Sec. 2.3: out(i, c) = v(i, c) * d_i^power with the
+ * context's current d (power = -0.5: Markov right eigenvectors from symmetric ones). */
+fd_status fd_scale_by_degree(fd_ctx* ctx, const float* v_dev, int64_t ldv, int32_t cols,
+                             double power, float* out_dev, int64_t ldout);
+
+const char* fd_status_string(fd_status st);
+const char* fd_last_error(const fd_ctx* ctx);
+int32_t     fd_version(void);
+/* Number of kernels this library has launched in the calling process (all contexts). */
+int64_t     fd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FD_H_ */
