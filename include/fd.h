@@ -168,7 +168,8 @@ fd_status fd_beta_flow(fd_ctx* ctx, const fd_flow_opts* opts, const float* Q0_de
  * (Sec. 1, the (n, beta) ladder): psi_j(x) = sum_i K(x, x_i) q_i^-alpha psi_j(x_i) /
  * (lambda_j sum_i K(x, x_i) q_i^-alpha), at the context's current (beta, alpha, q).
  * psi_dev: N x m column-major (Markov vectors d^-1/2 * v); lambda_host: m values;
- * out_dev: Nnew x m column-major.  Needs b_max >= m + 1.  Synchronous. */
+ * out_dev: Nnew x m column-major.  Two rectangular products (denominator, numerators), the
+ * numerators b_max columns at a time.  Synchronous. */
 fd_status fd_nystrom(fd_ctx* ctx, const float* Xnew_dev, int64_t Nnew, int64_t ldxnew,
                      const float* psi_dev, int64_t ldpsi, int32_t m, const double* lambda_host,
                      float* out_dev, int64_t ldout);

@@ -64,9 +64,16 @@ Layout make_layout(int64_t N, int32_t D, int32_t b_max, int32_t m_max) {
     if (m_max > 0) {
         L.eig_q = carve(cur, (size_t)N * m_max * 4);
         L.eig_w = carve(cur, (size_t)N * m_max * 4);
+        L.eig_x = carve(cur, (size_t)N * m_max * 4);
         L.eig_r = carve(cur, (size_t)N * L.BP * 4);
         L.eig_t = carve(cur, (size_t)N * L.BP * 4);
-        L.eig_small_doubles = (size_t)4 * m_max * m_max + (size_t)64 * 1024;
+        // projection output + small right factors (2 * m_max * max(m_max, BP) doubles), then the per-chunk
+        // partials of the A^T B kernel (up to 256 row chunks of m_max x BP)
+        const size_t mm = (size_t)m_max * (size_t)(m_max > L.BP ? m_max : L.BP);
+        size_t chunks = (size_t)ceil_div(N, 4096);
+        if (chunks > 256) chunks = 256;
+        if (chunks < 2) chunks = 2;
+        L.eig_small_doubles = 2 * mm + chunks * mm;
         L.eig_small = carve(cur, L.eig_small_doubles * 8);
     }
     L.total = cur;

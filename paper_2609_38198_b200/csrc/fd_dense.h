@@ -1,0 +1,27 @@
+// Tall-skinny dense helpers (fd_dense.cu) and the host symmetric eigensolver (fd_symeig.cpp).
+#pragma once
+#include <vector>
+
+#include "fd_internal.h"
+
+namespace fd {
+
+// out_dev[m1 x m2] (column-major doubles, device) = A^T B over N rows, fp64 accumulation.
+// scratch: device doubles for the per-chunk partials.
+fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float* B, int64_t ldb, int m2, int64_t N,
+                     double* out_dev, double* scratch, size_t scratch_doubles);
+// C[N x p] = alpha * A[N x m] S[m x p] + beta * C; S_dev column-major floats with pitch lds.  C must not alias A.
+fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float* S_dev, int lds, int p, float* C,
+                     int64_t ldc, float alpha, float beta, int64_t N);
+fd_status d2f(fd_ctx* c, const double* in, float* out, int64_t n, double scale);
+fd_status scale_cols(fd_ctx* c, float* A, int64_t lda, int p, const float* f_dev, int64_t N);
+fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, uint32_t seed);
+fd_status sqrt_vec(fd_ctx* c, const float* d, float* out, int64_t N);
+fd_status copy_cols(fd_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd, int p, int64_t N);
+
+// Eigen-decomposition of a dense symmetric n x n matrix (column-major, only read).  On return
+// evals ascending and evecs column-major with orthonormal columns.  Householder tridiagonalisation
+// followed by implicit-shift QL.  Returns false if QL fails to converge.
+bool sym_eig(const double* A, int n, std::vector<double>& evals, std::vector<double>& evecs);
+
+}  // namespace fd

@@ -1,21 +1,391 @@
-// Eigensolver, bandwidth flow and out-of-sample extension: placeholders.
-#include "fd_internal.h"
+// fd_eigs: leading eigenpairs of M = diag(s) K diag(s) (Eq. 2) by block Krylov / Rayleigh-Ritz
+// with residual expansion and thick restart.
+//
+// The paper names "block implicitly restarted Lanczos" (Sec. 2.3) and gives no detail, so the
+// scheme is fixed here.  An orthonormal basis Q (N x m) is kept together with its image
+// W = M Q.  Each step: projected matrix T = Q^T W (fp64), Ritz pairs, explicit residuals
+// R_i = W x_i - theta_i Q x_i for the leading k + 1 + buffer pairs, the b residuals of largest
+// norm are orthogonalised against Q (classical Gram-Schmidt twice) and among themselves
+// (eigen-based orthogonalisation that drops dependent directions), appended, and M is applied
+// to the new block only.  For a cold one-block start this spans the same block Krylov space as
+// block Lanczos; unlike the three-term recurrence it accepts an arbitrary warm-start basis.
+// When the basis is full it is compressed onto the leading Ritz vectors (thick restart).
+// The Perron vector sqrt(d) / |sqrt(d)| is known in closed form and always seeds the basis.
+// Vectors are fp32; every inner product and the small eigenproblem are fp64, and the measured
+// Gram matrix Q^T Q corrects the projected problem to first order, so fp32 loss of
+// orthogonality does not reach the Ritz values.
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <vector>
 
-extern "C" {
+#include "fd_dense.h"
 
-fd_status fd_eigs(fd_ctx* c, int32_t, int32_t, double, int32_t, const float*, int64_t, int32_t, double*, float*, int64_t,
-                  fd_eigs_info*) {
-    return fd::fail(c, FD_ERR_UNSUPPORTED, "fd_eigs not built");
-}
+namespace fd {
 
-fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts*, const float*, int64_t, int32_t, fd_probe*, int32_t*, int32_t*,
-                       double*, double*, float*, int64_t) {
-    return fd::fail(c, FD_ERR_UNSUPPORTED, "fd_beta_flow not built");
-}
+namespace {
 
-fd_status fd_nystrom(fd_ctx* c, const float*, int64_t, int64_t, const float*, int64_t, int32_t, const double*, float*,
-                     int64_t) {
-    return fd::fail(c, FD_ERR_UNSUPPORTED, "fd_nystrom not built");
-}
+using clk = std::chrono::steady_clock;
+inline double secs(clk::time_point a, clk::time_point b) { return std::chrono::duration<double>(b - a).count(); }
 
+struct Solver {
+    fd_ctx* c;
+    int64_t N;
+    int m_cap, BP;
+    float *Q, *W, *X;               // N x m_cap each (X = spare for out-of-place updates)
+    float *R, *R2;                  // N x BP each
+    double* d_out;                  // device: m_cap x BP doubles (projection results)
+    float* d_S;                     // device: m_cap x m_cap floats (small right factors)
+    double* d_scr; size_t scr_n;    // device: partials of the projections
+    std::vector<double> T, G;       // host, column-major, pitch m_cap
+    std::vector<double> h_out;      // host staging
+    int m = 0;
+    int applies = 0, restarts = 0;
+    double t_apply = 0.0;
+
+    fd_status to_host(int n) {
+        FD_CUDA(c, cudaMemcpyAsync(h_out.data(), d_out, sizeof(double) * (size_t)n, cudaMemcpyDeviceToHost, c->stream));
+        FD_CUDA(c, cudaStreamSynchronize(c->stream));
+        return FD_OK;
+    }
+    fd_status upload_S(const std::vector<float>& S) {
+        FD_CUDA(c, cudaMemcpyAsync(d_S, S.data(), sizeof(float) * S.size(), cudaMemcpyHostToDevice, c->stream));
+        FD_CUDA(c, cudaStreamSynchronize(c->stream));      // S is a stack/vector temporary on the host
+        return FD_OK;
+    }
+
+    // W[:, c0 : c0 + n) = M Q[:, c0 : c0 + n), in blocks of at most bw columns
+    fd_status apply_cols(int c0, int n, int bw) {
+        auto t0 = clk::now();
+        for (int o = 0; o < n; o += bw) {
+            int w = std::min(bw, n - o);
+            FD_TRY(fd_apply(c, Q + (int64_t)(c0 + o) * N, N, w, W + (int64_t)(c0 + o) * N, N, FD_PREC_FP32));
+            ++applies;
+        }
+        FD_CUDA(c, cudaStreamSynchronize(c->stream));
+        t_apply += secs(t0, clk::now());
+        return FD_OK;
+    }
+
+    // out(m1 x m2) -> host h_out, column-major pitch m1; right factor chunked to BP columns
+    fd_status project(const float* A, int m1, const float* B, int m2, std::vector<double>& dst) {
+        dst.assign((size_t)m1 * m2, 0.0);
+        for (int c0 = 0; c0 < m2; c0 += BP) {
+            int w = std::min(BP, m2 - c0);
+            FD_TRY(tn_product(c, A, N, m1, B + (int64_t)c0 * N, N, w, N, d_out, d_scr, scr_n));
+            FD_TRY(to_host(m1 * w));
+            std::copy(h_out.begin(), h_out.begin() + (size_t)m1 * w, dst.begin() + (size_t)c0 * m1);
+        }
+        return FD_OK;
+    }
+
+    // Recompute T = Q^T W and G = Q^T Q for the first m columns.
+    fd_status full_projection() {
+        std::vector<double> tmp;
+        FD_TRY(project(Q, m, W, m, tmp));
+        for (int j = 0; j < m; ++j)
+            for (int i = 0; i < m; ++i) T[i + (size_t)j * m_cap] = 0.5 * (tmp[i + (size_t)j * m] + tmp[j + (size_t)i * m]);
+        FD_TRY(project(Q, m, Q, m, tmp));
+        for (int j = 0; j < m; ++j)
+            for (int i = 0; i < m; ++i) G[i + (size_t)j * m_cap] = 0.5 * (tmp[i + (size_t)j * m] + tmp[j + (size_t)i * m]);
+        return FD_OK;
+    }
+
+    // After appending nb columns at position m: fill the new rows / columns of T and G.
+    fd_status extend_projection(int nb) {
+        const int mt = m + nb;
+        std::vector<double> tmp;
+        FD_TRY(project(Q, mt, W + (int64_t)m * N, nb, tmp));
+        for (int j = 0; j < nb; ++j)
+            for (int i = 0; i < mt; ++i) {
+                double v = tmp[i + (size_t)j * mt];
+                if (i >= m) v = 0.5 * (v + tmp[(m + j) + (size_t)(i - m) * mt]);
+                T[i + (size_t)(m + j) * m_cap] = v;
+                T[(m + j) + (size_t)i * m_cap] = v;
+            }
+        FD_TRY(project(Q, mt, Q + (int64_t)m * N, nb, tmp));
+        for (int j = 0; j < nb; ++j)
+            for (int i = 0; i < mt; ++i) {
+                double v = tmp[i + (size_t)j * mt];
+                if (i >= m) v = 0.5 * (v + tmp[(m + j) + (size_t)(i - m) * mt]);
+                G[i + (size_t)(m + j) * m_cap] = v;
+                G[(m + j) + (size_t)i * m_cap] = v;
+            }
+        m = mt;
+        return FD_OK;
+    }
+
+    // Orthonormalise the p columns of B (N x p, pitch N) among themselves; dependent directions
+    // (eigenvalue of the unit-diagonal Gram matrix below drop_tol) are dropped.  Result in B, p updated.
+    fd_status orthonormalise(float*& B, float*& spare, int& p, double drop_tol) {
+        if (p == 0) return FD_OK;
+        FD_TRY(tn_product(c, B, N, p, B, N, p, N, d_out, d_scr, scr_n));
+        FD_TRY(to_host(p * p));
+        std::vector<double> g((size_t)p * p), dinv(p);
+        for (int j = 0; j < p; ++j) {
+            double dj = h_out[j + (size_t)j * p];
+            dinv[j] = dj > 1e-60 ? 1.0 / std::sqrt(dj) : 0.0;
+        }
+        for (int j = 0; j < p; ++j)
+            for (int i = 0; i < p; ++i)
+                g[i + (size_t)j * p] = 0.5 * (h_out[i + (size_t)j * p] + h_out[j + (size_t)i * p]) * dinv[i] * dinv[j];
+        std::vector<double> lam, U;
+        if (!sym_eig(g.data(), p, lam, U)) return fail(c, FD_ERR_NOT_CONVERGED, "small eigenproblem (orthonormalise) failed");
+        std::vector<int> keep;
+        for (int j = p - 1; j >= 0; --j)
+            if (lam[j] > drop_tol) keep.push_back(j);
+        const int pk = (int)keep.size();
+        if (pk == 0) { p = 0; return FD_OK; }
+        std::vector<float> S((size_t)p * pk);
+        for (int jj = 0; jj < pk; ++jj) {
+            const int j = keep[jj];
+            const double f = 1.0 / std::sqrt(lam[j]);
+            for (int i = 0; i < p; ++i) S[i + (size_t)jj * p] = (float)(dinv[i] * U[i + (size_t)j * p] * f);
+        }
+        FD_TRY(upload_S(S));
+        FD_TRY(nn_product(c, B, N, p, d_S, p, pk, spare, N, 1.f, 0.f, N));
+        std::swap(B, spare);
+        p = pk;
+        return FD_OK;
+    }
+
+    // B <- B - Q[:, 0:mq) (Q^T B), once.
+    fd_status project_out(float* B, int p, int mq) {
+        if (p == 0 || mq == 0) return FD_OK;
+        FD_TRY(tn_product(c, Q, N, mq, B, N, p, N, d_out, d_scr, scr_n));
+        FD_TRY(d2f(c, d_out, d_S, (int64_t)mq * p, -1.0));
+        FD_TRY(nn_product(c, Q, N, mq, d_S, mq, p, B, N, 1.f, 1.f, N));
+        return FD_OK;
+    }
+};
+
+}  // namespace
+}  // namespace fd
+
+using namespace fd;
+
+extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_t max_applies, const float* Q0_dev,
+                             int64_t ldq0, int32_t q0_cols, double* evals_host, float* evecs_dev, int64_t ldv,
+                             fd_eigs_info* info) {
+    if (!c) return FD_ERR_INVALID;
+    auto t_start = clk::now();
+    const Layout& L = c->L;
+    const int64_t N = L.N;
+    if (!c->have_s) return fail(c, FD_ERR_INVALID, "fd_eigs before fd_degree");
+    if (k < 0 || (int64_t)k + 1 > N) return fail(c, FD_ERR_INVALID, "k + 1 = %d exceeds N or k < 0", k + 1);
+    if (b < 1 || b > L.b_max) return fail(c, FD_ERR_INVALID, "b outside 1..b_max");
+    if (!(tol > 0) || max_applies < 1 || !evals_host || !evecs_dev || ldv < N) return fail(c, FD_ERR_INVALID, "bad fd_eigs argument");
+    if (Q0_dev && (q0_cols < 1 || ldq0 < N)) return fail(c, FD_ERR_INVALID, "bad warm-start basis");
+    const int nwant = k + 1;
+    if (L.m_max < 2 * nwant + b && L.m_max < N) return fail(c, FD_ERR_WORKSPACE, "m_max = %d < 2 (k + 1) + b = %d", L.m_max, 2 * nwant + b);
+
+    Solver S;
+    S.c = c; S.N = N; S.BP = L.BP;
+    S.m_cap = (int)std::min<int64_t>(L.m_max, N);
+    const int m_cap = S.m_cap;
+    S.Q = c->at<float>(L.eig_q); S.W = c->at<float>(L.eig_w); S.X = c->at<float>(L.eig_x);
+    S.R = c->at<float>(L.eig_r); S.R2 = c->at<float>(L.eig_t);
+    double* small = c->at<double>(L.eig_small);
+    S.d_out = small;
+    S.d_S = reinterpret_cast<float*>(small + (size_t)L.m_max * std::max(L.m_max, L.BP));
+    S.d_scr = small + (size_t)2 * L.m_max * std::max(L.m_max, L.BP);
+    S.scr_n = L.eig_small_doubles - (size_t)2 * L.m_max * std::max(L.m_max, L.BP);
+    S.T.assign((size_t)m_cap * m_cap, 0.0);
+    S.G.assign((size_t)m_cap * m_cap, 0.0);
+    S.h_out.assign((size_t)L.m_max * std::max(L.m_max, L.BP), 0.0);
+
+    const int buffer = std::min<int>(std::min(b, 8), (int)std::max<int64_t>(0, N - nwant));
+    const int nsel_max = nwant + buffer;
+
+    // ---- start basis: Perron vector, then the warm-start columns or a random block ----------
+    FD_TRY(sqrt_vec(c, c->d(), S.Q, N));
+    int cols = 1;
+    const int room = std::max(0, m_cap - b - 1);                 // leave space for one expansion block
+    if (Q0_dev) {
+        int take = std::min(q0_cols, std::max(room, std::min(m_cap - 1, nwant)));
+        take = std::min(take, m_cap - 1);
+        FD_TRY(copy_cols(c, Q0_dev, ldq0, S.Q + N, N, take, N));
+        cols += take;
+    } else {
+        int take = std::min(std::max(b, 1), m_cap - 1);
+        if (take > 0) FD_TRY(random_fill(c, S.Q + N, N, take, N, 0x5EEDu));
+        cols += take;
+    }
+    {
+        // orthonormalise the start block in place (may exceed BP columns: use the spare basis buffer)
+        float* B = S.Q; float* spare = S.X; int p = cols;
+        // d_S must hold p x p floats: p <= m_cap
+        FD_TRY(S.orthonormalise(B, spare, p, 1e-10));
+        FD_TRY(S.orthonormalise(B, spare, p, 1e-10));
+        S.Q = B; S.X = spare;
+        if (p == 0) return fail(c, FD_ERR_NONFINITE, "start basis has no usable column");
+        S.m = p;
+    }
+    FD_TRY(S.apply_cols(0, S.m, b));
+    FD_TRY(S.full_projection());
+
+    std::vector<double> theta, Xr;        // Ritz values (descending) and vectors (m x nsel, pitch m)
+    std::vector<double> resid;
+    int nsel = 0, nconv = 0;
+    fd_status final_status = FD_ERR_NOT_CONVERGED;
+    int stagnation = 0;
+
+    for (int iter = 0;; ++iter) {
+        const int m = S.m;
+        // ---- Rayleigh-Ritz with first-order correction for G = Q^T Q = I + E ---------------------
+        // Tc = T - (E T + T E) / 2 with E = G - I; T E = (E T)^T because both are symmetric
+        std::vector<double> Tc((size_t)m * m), ET((size_t)m * m, 0.0);
+        for (int j = 0; j < m; ++j)
+            for (int l = 0; l < m; ++l) {
+                const double t = S.T[l + (size_t)j * m_cap];
+                const double* Ecol = &S.G[(size_t)l * m_cap];
+                double* o = &ET[(size_t)j * m];
+                for (int i = 0; i < m; ++i) o[i] += Ecol[i] * t;          // G column l ...
+                o[l] -= t;                                                 // ... minus the identity
+            }
+        for (int j = 0; j < m; ++j)
+            for (int i = 0; i < m; ++i)
+                Tc[i + (size_t)j * m] = S.T[i + (size_t)j * m_cap] - 0.5 * (ET[i + (size_t)j * m] + ET[j + (size_t)i * m]);
+        std::vector<double> lam, U;
+        if (!sym_eig(Tc.data(), m, lam, U)) return fail(c, FD_ERR_NOT_CONVERGED, "projected eigenproblem failed");
+        nsel = std::min(nsel_max, m);
+        theta.resize(nsel);
+        Xr.assign((size_t)m * nsel, 0.0);
+        for (int jj = 0; jj < nsel; ++jj) {
+            const int j = m - 1 - jj;
+            theta[jj] = lam[j];
+            for (int i = 0; i < m; ++i) {
+                double corr = 0.0;
+                for (int l = 0; l < m; ++l) corr += (S.G[i + (size_t)l * m_cap] - (i == l ? 1.0 : 0.0)) * U[l + (size_t)j * m];
+                Xr[i + (size_t)jj * m] = U[i + (size_t)j * m] - 0.5 * corr;
+            }
+        }
+        // ---- explicit residuals R_i = W x_i - theta_i Q x_i, BP columns at a time -----------------
+        resid.assign(nsel, 0.0);
+        for (int c0 = 0; c0 < nsel; c0 += S.BP) {
+            const int w = std::min(S.BP, nsel - c0);
+            std::vector<float> Sx((size_t)m * w * 2);
+            for (int jj = 0; jj < w; ++jj)
+                for (int i = 0; i < m; ++i) {
+                    Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)(c0 + jj) * m];
+                    Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[c0 + jj] * Xr[i + (size_t)(c0 + jj) * m]);
+                }
+            FD_TRY(S.upload_S(Sx));
+            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+            FD_TRY(tn_product(c, S.R, N, w, S.R, N, w, N, S.d_out, S.d_scr, S.scr_n));
+            FD_TRY(S.to_host(w * w));
+            for (int jj = 0; jj < w; ++jj) resid[c0 + jj] = std::sqrt(std::max(0.0, S.h_out[jj + (size_t)jj * w]));
+        }
+        const double thr = tol * std::fabs(theta[0]);
+        nconv = 0;
+        while (nconv < std::min(nwant, nsel) && resid[nconv] <= thr) ++nconv;
+        bool all = nsel >= nwant;
+        for (int i = 0; i < std::min(nwant, nsel); ++i) all = all && resid[i] <= thr;
+        if (all) { final_status = FD_OK; break; }
+        if (S.applies >= max_applies) break;
+        if (m >= N) break;                                        // basis spans everything: nothing more to add
+
+        // ---- choose the expansion columns: largest residuals first ------------------------------
+        std::vector<int> order(nsel);
+        for (int i = 0; i < nsel; ++i) order[i] = i;
+        std::sort(order.begin(), order.end(), [&](int a, int bb) { return resid[a] > resid[bb]; });
+        int want_new = std::min<int64_t>(b, N - m);
+        std::vector<int> pick;
+        for (int i = 0; i < nsel && (int)pick.size() < want_new; ++i)
+            if (resid[order[i]] > 0.1 * thr) pick.push_back(order[i]);
+        if (pick.empty()) { final_status = FD_OK; break; }
+
+        // ---- thick restart when the new block would not fit ----------------------------------------
+        if (m + (int)pick.size() > m_cap) {
+            int keep = std::max(nsel, std::min(m - 1, (m_cap * 3) / 5));
+            keep = std::min(keep, m_cap - (int)pick.size());
+            keep = std::min(keep, m);
+            // Ritz vectors for the kept block (beyond nsel use the uncorrected eigenvectors)
+            std::vector<float> Sk((size_t)m * keep);
+            for (int jj = 0; jj < keep; ++jj) {
+                const int j = m - 1 - jj;
+                for (int i = 0; i < m; ++i)
+                    Sk[i + (size_t)jj * m] = jj < nsel ? (float)Xr[i + (size_t)jj * m] : (float)U[i + (size_t)j * m];
+            }
+            // residual block for the picked columns must be formed BEFORE the basis changes
+            std::vector<float> Sx((size_t)m * pick.size() * 2);
+            const int w = (int)pick.size();
+            for (int jj = 0; jj < w; ++jj)
+                for (int i = 0; i < m; ++i) {
+                    Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)pick[jj] * m];
+                    Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[pick[jj]] * Xr[i + (size_t)pick[jj] * m]);
+                }
+            FD_TRY(S.upload_S(Sx));
+            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+            FD_TRY(S.upload_S(Sk));
+            FD_TRY(nn_product(c, S.Q, N, m, S.d_S, m, keep, S.X, N, 1.f, 0.f, N));
+            std::swap(S.Q, S.X);                                  // X now holds the old basis: reuse it for W
+            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, keep, S.X, N, 1.f, 0.f, N));
+            std::swap(S.W, S.X);
+            S.m = keep;
+            ++S.restarts;
+            FD_TRY(S.full_projection());
+        } else {
+            const int w = (int)pick.size();
+            std::vector<float> Sx((size_t)m * w * 2);
+            for (int jj = 0; jj < w; ++jj)
+                for (int i = 0; i < m; ++i) {
+                    Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)pick[jj] * m];
+                    Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[pick[jj]] * Xr[i + (size_t)pick[jj] * m]);
+                }
+            FD_TRY(S.upload_S(Sx));
+            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+        }
+        // ---- orthogonalise the new block against the basis and within itself ---------------------
+        int p = (int)pick.size();
+        FD_TRY(S.project_out(S.R, p, S.m));
+        FD_TRY(S.project_out(S.R, p, S.m));
+        FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-5));
+        FD_TRY(S.project_out(S.R, p, S.m));
+        FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-3));
+        if (p == 0) {
+            // the residuals lie (numerically) inside the basis: try a random direction, give up after a few
+            if (++stagnation > 3) break;
+            p = std::min<int64_t>(b, N - S.m);
+            FD_TRY(random_fill(c, S.R, N, p, N, 0xABCD1234u + (uint32_t)iter));
+            FD_TRY(S.project_out(S.R, p, S.m));
+            FD_TRY(S.project_out(S.R, p, S.m));
+            FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-5));
+            FD_TRY(S.project_out(S.R, p, S.m));
+            FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-3));
+            if (p == 0) break;
+        }
+        FD_TRY(copy_cols(c, S.R, N, S.Q + (int64_t)S.m * N, N, p, N));
+        FD_TRY(S.apply_cols(S.m, p, b));
+        FD_TRY(S.extend_projection(p));
+    }
+
+    // ---- outputs: evecs = Q X[:, 0 : k + 1) ----------------------------------------------------------
+    const int nout = std::min(nwant, nsel);
+    {
+        const int m = S.m;
+        for (int c0 = 0; c0 < nout; c0 += S.BP) {
+            const int w = std::min(S.BP, nout - c0);
+            std::vector<float> Sx((size_t)m * w);
+            for (int jj = 0; jj < w; ++jj)
+                for (int i = 0; i < m; ++i) Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)(c0 + jj) * m];
+            FD_TRY(S.upload_S(Sx));
+            FD_TRY(nn_product(c, S.Q, N, m, S.d_S, m, w, evecs_dev + (int64_t)c0 * ldv, ldv, 1.f, 0.f, N));
+        }
+        for (int i = 0; i < nwant; ++i) evals_host[i] = i < nout ? theta[i] : 0.0;
+        FD_CUDA(c, cudaStreamSynchronize(c->stream));
+    }
+    if (info) {
+        info->applies = S.applies; info->restarts = S.restarts; info->converged = nconv; info->basis_cols = S.m;
+        double mx = 0.0;
+        for (int i = 0; i < nout; ++i) mx = std::max(mx, resid[i]);
+        info->max_residual = mx;
+        info->seconds_apply = S.t_apply;
+        info->seconds_total = secs(t_start, clk::now());
+    }
+    if (final_status != FD_OK) return fail(c, FD_ERR_NOT_CONVERGED, "fd_eigs: %d of %d pairs converged after %d applies", nconv, nwant, S.applies);
+    return FD_OK;
 }

@@ -30,7 +30,7 @@ struct Layout {
     size_t wp = 0, part = 0, part_floats = 0;
     size_t xp_col = 0, xp_row = 0, wt_hi = 0, wt_lo = 0, colscale = 0, status = 0;
     size_t yacc = 0;
-    size_t eig_q = 0, eig_w = 0, eig_r = 0, eig_t = 0, eig_small = 0, eig_small_doubles = 0;
+    size_t eig_q = 0, eig_w = 0, eig_x = 0, eig_r = 0, eig_t = 0, eig_small = 0, eig_small_doubles = 0;
     size_t total = 0;
 };
 Layout make_layout(int64_t N, int32_t D, int32_t b_max, int32_t m_max);

@@ -49,8 +49,9 @@ def run_case(fd, dev, X, beta, alpha, b, path, seed=1, prec=0, tol=TOL_APPLY):
     assert np.abs(q.cpu().numpy() / qo - 1).max() <= tol
     assert np.abs(d.cpu().numpy() / do - 1).max() <= 2 * tol
     assert np.abs(s.cpu().numpy() / s_o - 1).max() <= 2 * tol
-    assert abs(so - soo) <= max(1e-6, tol / 10) * max(soo, 1e-30) + 1e-9 * N
-    assert abs(so2 - so2o) <= max(1e-6, tol / 10) * max(so2o, 1e-30) + 1e-9 * N
+    # S_off = sum(q) - N with q held in fp32: absolute floor of ~1e-7 per row on top of the relative bound
+    assert abs(so - soo) <= max(1e-6, tol / 10) * soo + 2e-7 * N
+    assert abs(so2 - so2o) <= max(1e-6, tol / 10) * so2o + 2e-7 * N
     err = relF(Y.cpu().numpy(), Yo)
     assert err <= tol, f"apply rel-Frobenius error {err:.3e}"
     ctx.close()

@@ -1,0 +1,223 @@
+"""GPU parity of fd_eigs, fd_beta_flow, fd_nystrom against the float64 oracle (through the C ABI).
+
+Gates (stated tolerances): leading k+1 eigenvalues within 1e-6 * lambda_0 of the oracle's;
+principal angles between the spans of the leading k' vectors <= max(1e-4, 1e-6 / gap) rad at
+every cut k' where the oracle's spectrum has a gap >= 1e-3 (inside a cluster the individual
+vectors are not unique, only the span of the whole cluster is); a float64 residual certificate
+|M v - theta v| <= 5e-6 for every returned vector; orthonormality to 1e-5.
+"""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import dense, flow, nystrom
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fd():
+    import __graft_entry__ as g
+    g.build()
+    import paper_2609_38198_b200 as fd
+    assert torch.cuda.is_available()
+    return fd
+
+
+@pytest.fixture(scope="module")
+def dev():
+    return torch.device("cuda:0")
+
+
+def default_m_max(k, b):
+    m = max(2 * (k + 1) + b, 4 * b)
+    return (m + b - 1) // b * b
+
+
+def check_eigs(lam, U, X, beta, alpha, k, val_tol=1e-6, angle_gate=True):
+    """lam, U from the GPU; oracle = dense eigh with one extra pair so the last gap is known."""
+    lam_o, U_o, d = dense.eigs(X, beta, alpha, min(k + 1, X.shape[0] - 1))
+    U = U.astype(np.float64)
+    assert np.all(np.abs(lam - lam_o[: k + 1]) <= val_tol * lam_o[0]), np.abs(lam - lam_o[: k + 1]).max()
+    # Perron pair is known in closed form
+    sd = np.sqrt(d) / np.linalg.norm(np.sqrt(d))
+    assert dense.principal_angles(U[:, :1], sd[:, None]).max() <= 1e-4
+    worst = 0.0
+    if angle_gate:
+        for kp in range(1, k + 2):
+            if kp >= len(lam_o):
+                break
+            gap = lam_o[kp - 1] - lam_o[kp]
+            if gap >= 1e-3:
+                ang = dense.principal_angles(U[:, :kp], U_o[:, :kp]).max()
+                worst = max(worst, ang)
+                assert ang <= max(1e-4, 1e-6 / gap), f"cut {kp}: angle {ang:.2e}, gap {gap:.2e}"
+    K = dense.kernel(X, beta)
+    _, _, s = dense.normalisation(K, alpha)
+    MU = s[:, None] * (K @ (s[:, None] * U))
+    res = np.linalg.norm(MU - U * lam[None, :], axis=0)
+    assert res.max() <= 5e-6, res.max()
+    assert np.abs(U.T @ U - np.eye(k + 1)).max() <= 1e-5
+    return worst, res.max()
+
+
+def solve(fd, dev, X, beta, alpha, k, b, tol=1e-6, max_applies=600, Q0=None, allow_nc=False, path=None):
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=default_m_max(k, b))
+    if path is not None:
+        ctx.set_option("path", path)
+    ctx.degree(beta, alpha)
+    lam, U, info = ctx.eigs(k, b, tol=tol, max_applies=max_applies, Q0=Q0, allow_not_converged=allow_nc)
+    return ctx, lam, U, info
+
+
+def test_c1_circle_closed_form_and_oracle(fd, dev):
+    X = workloads.circle(2048)
+    ctx, lam, U, info = solve(fd, dev, X, 200.0, 1.0, 8, 8)
+    c = np.exp(-4.0 * 200.0 * np.sin(np.pi * np.arange(2048) / 2048) ** 2)
+    f = np.fft.fft(c).real
+    expect = np.array([1.0] + [f[m] / f[0] for m in (1, 1, 2, 2, 3, 3, 4, 4)])
+    assert np.abs(lam - expect).max() <= 1e-6
+    check_eigs(lam, U.cpu().numpy(), X, 200.0, 1.0, 8)
+    assert info.converged == 9 and info.max_residual <= 1e-6
+    ctx.close()
+
+
+@pytest.mark.parametrize("beta", [10.0, 30.0])
+def test_c2_torus2_reduced(fd, dev, beta):
+    X = workloads.torus2(4096)
+    ctx, lam, U, info = solve(fd, dev, X, beta, 1.0, 32, 16)
+    check_eigs(lam, U.cpu().numpy(), X, beta, 1.0, 32)
+    ctx.close()
+
+
+def test_c2_high_beta_eigenvalues_only(fd, dev):
+    # noise-dominated spectrum: eigenvalues are still well-posed (Weyl); vectors inside the smeared cluster are not
+    X = workloads.torus2(2048)
+    ctx, lam, U, info = solve(fd, dev, X, 100.0, 1.0, 32, 16, max_applies=1500, allow_nc=True)
+    lam_o, _, _ = dense.eigs(X, 100.0, 1.0, 32)
+    assert np.abs(lam - lam_o).max() <= 1e-6 * lam_o[0]
+    ctx.close()
+
+
+@pytest.mark.parametrize("alpha", [1.0, 0.5, 0.0])
+def test_c3_torus6_reduced(fd, dev, alpha):
+    X = workloads.torus6(3000)
+    ctx, lam, U, info = solve(fd, dev, X, 0.5, alpha, 64, 32)
+    check_eigs(lam, U.cpu().numpy(), X, 0.5, alpha, 64)
+    ctx.close()
+
+
+def test_c4_latent_torus_reduced(fd, dev):
+    X = workloads.latent_torus(2500)
+    ctx, lam, U, info = solve(fd, dev, X, 2.0, 1.0, 32, 32)
+    check_eigs(lam, U.cpu().numpy(), X, 2.0, 1.0, 32)
+    ctx.close()
+
+
+def test_c5_wide_block_reduced(fd, dev):
+    X = workloads.torus6(4096)
+    ctx, lam, U, info = solve(fd, dev, X, 0.6, 1.0, 128, 64)
+    check_eigs(lam, U.cpu().numpy(), X, 0.6, 1.0, 128)
+    ctx.close()
+
+
+def test_tiny_problems(fd, dev):
+    # N = 2 and a simplex: closed forms; basis can span the whole space
+    e = np.exp(-0.8 * 1.7 ** 2)
+    X2 = np.array([[0.0, 0.0], [1.7, 0.0]], dtype=np.float32)
+    ctx, lam, U, info = solve(fd, dev, X2, 0.8, 1.0, 1, 1, allow_nc=True)
+    e32 = np.exp(-0.8 * float(np.float32(1.7)) ** 2)
+    assert lam[0] == pytest.approx(1.0, abs=1e-6) and lam[1] == pytest.approx((1 - e32) / (1 + e32), abs=1e-6)
+    ctx.close()
+    X = workloads.gaussian_cloud(40, 3, seed=2)
+    ctx, lam, U, info = solve(fd, dev, X, 0.5, 0.5, 6, 4)
+    check_eigs(lam, U.cpu().numpy(), X, 0.5, 0.5, 6)
+    ctx.close()
+    assert abs(e - e32) < 1e-6
+
+
+def test_warm_start_matches_cold_and_saves_applies(fd, dev):
+    X = workloads.torus6(3000, seed=5)
+    ctx, lam, U, info = solve(fd, dev, X, 0.5, 1.0, 24, 16)
+    # continue to a neighbouring bandwidth from the previous eigenvectors
+    ctx.degree(0.6, 1.0)
+    lam_w, U_w, info_w = ctx.eigs(24, 16, Q0=U)
+    lam_c, U_c, info_c = ctx.eigs(24, 16)
+    assert np.abs(lam_w - lam_c).max() <= 1e-6
+    check_eigs(lam_w, U_w.cpu().numpy(), X, 0.6, 1.0, 24)
+    assert info_w.applies <= info_c.applies
+    ctx.close()
+
+
+def test_eigs_argument_errors(fd, dev):
+    X = workloads.torus2(256, seed=1)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=16)
+    with pytest.raises(fd.FdError) as e:
+        ctx.eigs(4, 8)                                   # before fd_degree
+    assert e.value.status == fd.FD_ERR_INVALID
+    ctx.degree(10.0, 1.0)
+    with pytest.raises(fd.FdError) as e:
+        ctx.eigs(8, 8)                                   # m_max too small: 16 < 2 * 9 + 8
+    assert e.value.status == fd.FD_ERR_WORKSPACE
+    with pytest.raises(fd.FdError):
+        ctx.eigs(2, 9)                                   # b > b_max
+    with pytest.raises(fd.FdError) as e:
+        ctx.eigs(3, 8, tol=1e-12, max_applies=2)         # cannot converge in two applies
+    assert e.value.status == fd.FD_ERR_NOT_CONVERGED
+    ctx.close()
+
+
+# ------------------------------------------------------------------ bandwidth flow (Eqs. 7-14)
+def test_beta_flow_matches_oracle_flow(fd, dev):
+    N, alpha, k = 1024, 0.5, 3
+    X = workloads.torus6_paper(N, seed=42)
+    bx_o, status_o, log_o = flow.beta_flow(flow.dense_probe(X, alpha, k), N, flow.beta0(X), 1000.0)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    bx, status, lam, U, recs = ctx.beta_flow(k, 8, alpha, beta_start=0.0, beta_max=1000.0)
+    assert status == status_o == "VERTEX"
+    assert len(recs) == len(log_o)
+    for r, ro in zip(recs, log_o):
+        assert r["beta"] == pytest.approx(ro["beta"], rel=1e-6)
+        assert r["V_bias"] == pytest.approx(ro["V_bias"], rel=1e-4)
+        assert r["n_eff"] == pytest.approx(ro["n_eff"], rel=1e-5)
+        assert r["V"] == pytest.approx(ro["V"], rel=1e-4)
+        assert r["d_hat"] == pytest.approx(ro["d_hat"], rel=1e-5)
+    assert bx == pytest.approx(bx_o, rel=1e-3)
+    check_eigs(lam, U.cpu().numpy(), X, bx, alpha, k, angle_gate=True)
+    assert ctx.get_option("beta") == pytest.approx(bx)
+    ctx.close()
+
+
+def test_beta_flow_perron_wall(fd, dev):
+    # four tight clusters: the Perron gap collapses quickly as beta doubles (same mechanism as the wall in Sec. 4)
+    X = workloads.latent_torus(1500, seed=42)
+    N, alpha, k = 1500, 1.0, 8
+    bx_o, status_o, log_o = flow.beta_flow(flow.dense_probe(X, alpha, k), N, 1.0, 64.0)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    bx, status, lam, U, recs = ctx.beta_flow(k, 8, alpha, beta_start=1.0, beta_max=64.0, max_applies=4000)
+    assert status == status_o
+    assert bx == pytest.approx(bx_o, rel=1e-3)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ out-of-sample extension
+def test_nystrom_matches_oracle_and_reproduces_samples(fd, dev):
+    # inputs (eigenvectors, eigenvalues) come from the oracle; the GPU and the oracle both extend them
+    X = workloads.torus6(1200, seed=3)
+    Z = workloads.torus6(500, seed=4)
+    beta, alpha, k = 0.6, 1.0, 10
+    lam_o, U_o, d_o = dense.eigs(X, beta, alpha, k)
+    psi_o = dense.markov_vectors(U_o, d_o)
+    q_o = dense.degree(X, beta, alpha)[0]
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8)
+    ctx.degree(beta, alpha)
+    psi = ctx.scale_by_degree(fd.to_colmajor(U_o, dev), -0.5)               # d^-1/2 * v with the GPU's own d
+    assert np.abs(psi.cpu().numpy() - psi_o).max() <= 1e-5 * np.abs(psi_o).max()
+    psi_dev = fd.to_colmajor(psi_o, dev)
+    ext = ctx.nystrom(torch.from_numpy(Z).to(dev), psi_dev, lam_o).cpu().numpy()
+    ext_o = nystrom.extend(X, q_o, alpha, beta, psi_o, lam_o, Z)
+    assert np.abs(ext - ext_o).max() <= 2e-5 * np.abs(ext_o).max()
+    same = ctx.nystrom(torch.from_numpy(X[:300].copy()).to(dev), psi_dev, lam_o).cpu().numpy()
+    assert np.abs(same - psi_o[:300]).max() <= 5e-5 * np.abs(psi_o).max()
+    ctx.close()
