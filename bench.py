@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the FlashDiffusion hot path on B200.
+
+One step = one pass of the whole hot path at a fixed bandwidth over the headline workload
+(6-torus in R^12, N = 2^20, block b = 64, alpha = 1, beta = 2): degree pass q = K 1, second
+normalisation pass d = q^-a * K q^-a, scale vector s, and the block product Y = M V.  A step
+therefore processes (b + 2) N^2 pair-columns; `value` is that count over the step time,
+aggregated over ranks (each rank runs an independent replica: the path is not sharded).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--n LOG2N]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU float64 oracle on a bounded
+row sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "kernel-apply pair-columns per second (degree passes + block product, one step)"
+UNIT = "pair*cols/s"
+
+# Peaks for the roofline: MUFU 16 ex2/clk/SM, FMA pipe 128 FFMA/clk/SM, 148 SMs.
+SM_COUNT = 148
+MUFU_PER_CLK_SM = 16
+FMA_PER_CLK_SM = 128
+
+# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None.
+NCU_TRAFFIC_BYTES = {"simt": None, "tc": None}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.idx)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); smax.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "power_w_max": float(max(power)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload(log2n: int):
+    import workloads
+    N = 1 << log2n
+    X = workloads.torus6(N, seed=42)
+    V = workloads.block(N, 64, seed=1)
+    return X, V, dict(workload=f"C5: 6-torus R^12 + noise 0.01, N=2^{log2n}, b=64, alpha=1, beta=2.0",
+                      N=N, D=12, b=64, alpha=1.0, beta=2.0, l2_note="inputs (X, V, Y: >= 0.6 GB) exceed the 126 MB L2")
+
+
+# ------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_step(X64, V64, beta, alpha, rows, q_hint=None):
+    """One bounded sample of the step on the CPU oracle: the three passes on `rows` rows."""
+    from oracle import blocked
+    q_rows, _ = blocked.rows_apply_general(X64, beta, None, rows=rows, want_rowsq=True)
+    # the second pass and the product need q, s on all columns: use a positive surrogate vector of the right
+    # magnitude for the columns (the cost per pair is what is being timed, not the values)
+    w = q_hint
+    blocked.rows_apply_general(X64, beta, None, rows=rows, left=w, right=w)
+    blocked.rows_apply_general(X64, beta, V64, rows=rows, left=w, right=w)
+    return q_rows
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import blocked
+    X, V, cfg = workload(args.n)
+    N, b = cfg["N"], cfg["b"]
+    X64 = X.astype(np.float64)
+    V64 = np.ascontiguousarray(V.astype(np.float64))
+    cores = blocked.threads()
+    # size the sample for ~6-10 s per step on this host: ~4e7 pair-evaluations per core-second over three passes
+    rows_n = int(max(16, min(N, 6.0 * cores * 2.0e7 / N)))
+    import workloads
+    rows = workloads.row_sample(N, rows_n, seed=11)
+    w = np.full(N, 1e-2)
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows[: max(16, rows_n // 8)], w)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows, w)
+    dt = (time.perf_counter() - t0) / args.steps
+    units = rows_n * N * (b + 2)
+    value = units / dt
+    sample = f"{rows_n} sampled rows x all {N} columns, three passes (b = 1, 1, {b}), float64, rows.c + OpenMP"
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------- GPU arm
+def run_gpu(args):
+    import torch
+    import paper_2609_38198_b200 as fd
+    from paper_2609_38198_b200 import build as fd_build
+    fd_build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+
+    X, V, cfg = workload(args.n)
+    N, b, beta, alpha = cfg["N"], cfg["b"], cfg["beta"], cfg["alpha"]
+    Xh = torch.from_numpy(X).pin_memory()
+    Vh = torch.from_numpy(np.ascontiguousarray(V.T)).pin_memory()          # (b, N): column-major N x b
+    Yh = torch.empty((b, N), dtype=torch.float32).pin_memory()
+    Xd = Xh.to(dev)
+    Vd = Vh.to(dev).t()
+    Yd = torch.empty((b, N), dtype=torch.float32, device=dev).t()
+    ctx = fd.Context(Xd, b_max=b, m_max=0)
+    if args.path:
+        ctx.set_option("path", {"auto": 0, "simt": 1, "tc": 2}[args.path])
+    stream = torch.cuda.current_stream(dev)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(timers=None):
+        e0, e1, e2 = ev(), ev(), ev()
+        e0.record(stream)
+        ctx.degree(beta, alpha)
+        e1.record(stream)
+        ctx.apply(Vd, out=Yd)
+        e2.record(stream)
+        if timers is not None:
+            timers.append((e0, e1, e2))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    timers = []
+    launches0 = fd.fd_launch_count()
+    t_start, t_end = ev(), ev()
+    barrier()
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step(timers)
+    t_end.record(stream)
+    barrier()
+    launches = fd.fd_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_start.elapsed_time(t_end)
+    deg_ms = float(np.mean([a.elapsed_time(b_) for a, b_, _ in timers]))
+    app_ms = float(np.mean([b_.elapsed_time(c_) for _, b_, c_ in timers]))
+
+    # end-to-end through the public API with host buffers: H2D of X and V, D2H of Y every step
+    def e2e_step():
+        Xd.copy_(Xh, non_blocking=True)
+        Vd.t().copy_(Vh, non_blocking=True)
+        c2 = fd.Context(Xd, b_max=b, m_max=0)
+        if args.path:
+            c2.set_option("path", {"auto": 0, "simt": 1, "tc": 2}[args.path])
+        c2.degree(beta, alpha)
+        c2.apply(Vd, out=Yd)
+        Yh.copy_(Yd.t(), non_blocking=True)
+        torch.cuda.synchronize(dev)
+        c2.close()
+
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_step()
+    barrier()
+    e_a, e_b = ev(), ev()
+    e_a.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e_b.record(stream)
+    barrier()
+    e2e_ms = e_a.elapsed_time(e_b) / e2e_steps
+
+    t = torch.tensor([total_ms, e2e_ms, deg_ms, app_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms, deg_ms, app_ms = [float(v) for v in t.cpu()]
+    step_ms = total_ms / args.steps
+    units = float(N) * N * (b + 2)
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        path_used = "simt" if ctx.get_option("path") == 1 or not TC_BUILT(fd, ctx) else "tc"
+        pairs_per_s = float(N) * N / (app_ms * 1e-3)
+        mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
+        mufu_peak = SM_COUNT * MUFU_PER_CLK_SM * peaks.get("sm_max_mhz", 1965.0) * 1e6       # exp / s
+        fma_peak = SM_COUNT * FMA_PER_CLK_SM * peaks.get("sm_max_mhz", 1965.0) * 1e6         # FMA / s
+        D = cfg["D"]
+        if path_used == "simt":
+            # everything on the FMA pipe: per pair 2 D (difference form) + b (product) + ~3 issue slots
+            peak_pairs = fma_peak / (2 * D + b + 3)
+            binder = "fma_pipe (direct-difference distance + block product on FFMA)"
+        else:
+            peak_pairs = mufu_peak
+            binder = "mufu (one ex2 per pair)"
+        roofline = {"bound": "alu", "kernel": "block product Y = M V (dominant kernel)", "binder": binder,
+                    "achieved": pairs_per_s / 1e9, "peak": peak_pairs / 1e9, "unit": "Gpairs/s",
+                    "frac": pairs_per_s / peak_pairs, "peak_source": f"unit counts x {peak_kind} max SM clock",
+                    "mufu_floor_frac": pairs_per_s / mufu_peak, "traffic": NCU_TRAFFIC_BYTES.get(path_used),
+                    "sm_mhz_seen": mhz}
+        out = {"metric": METRIC, "value": units * world / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
+               "apply_only": {"ms": app_ms, "pair_cols_per_s": float(N) * N * b / (app_ms * 1e-3), "pairs_per_s": pairs_per_s},
+               "degree_ms": deg_ms, "path": path_used, "roofline": roofline,
+               "e2e": {"value": units * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": int(Xh.numel() * 4 + Vh.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 4)},
+               "gpu_launches": int(launches), "workspace_bytes": ctx.workspace_bytes}
+        if not args.no_cpu and world == 1 or (not args.no_cpu and rank == 0):
+            out["cpu_baseline"] = cpu_baseline(X, V, cfg)
+        print(json.dumps(out), flush=True)
+    ctx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def TC_BUILT(fd, ctx) -> bool:
+    """True when the tensor-core path serves this shape (probe by option)."""
+    try:
+        return bool(ctx.get_option("tc_active"))
+    except Exception:
+        return False
+
+
+def cpu_baseline(X, V, cfg):
+    from oracle import blocked
+    import workloads
+    N, b = cfg["N"], cfg["b"]
+    cores = blocked.threads()
+    rows_n = int(max(16, min(N, 12.0 * cores * 2.0e7 / N)))
+    rows = workloads.row_sample(N, rows_n, seed=11)
+    X64 = X.astype(np.float64)
+    V64 = np.ascontiguousarray(V.astype(np.float64))
+    w = np.full(N, 1e-2)
+    oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows[:16], w)
+    t0 = time.perf_counter()
+    oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows, w)
+    dt = time.perf_counter() - t0
+    return {"value": rows_n * float(N) * (b + 2) / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
+            "sample": f"{rows_n} sampled rows x all {N} columns, three passes (b = 1, 1, {b}), float64, rows.c + OpenMP"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=20, help="log2 of the number of points (default 20: the headline size)")
+    ap.add_argument("--path", default="", choices=["", "auto", "simt", "tc"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

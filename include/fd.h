@@ -80,8 +80,9 @@ fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int6
 fd_status fd_destroy(fd_ctx* ctx);
 
 /* Tuning / test knobs by name: "path" (FD_PATH_*), "splits" (0 = auto), "flush" (column tiles
- * between accumulator flushes of the tensor-core kernel), "poly_exp" (share of exponentials sent
- * to the FMA pipe, 0..1).  Unknown name -> FD_ERR_INVALID. */
+ * between accumulator flushes of the tensor-core kernel), "tc_max_mag" (largest beta * log2(e) *
+ * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "poly_exp" (share
+ * of exponentials sent to the FMA pipe, 0..1).  Unknown name -> FD_ERR_INVALID. */
 fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
 fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);
 
@@ -102,6 +103,11 @@ fd_status fd_degree(fd_ctx* ctx, double beta, double alpha, fd_precision prec,
  * V_dev and Y_dev must not overlap.  Asynchronous. */
 fd_status fd_apply(fd_ctx* ctx, const float* V_dev, int64_t ldv, int32_t b,
                    float* Y_dev, int64_t ldy, fd_precision prec);
+
+/* Waits for everything the context has enqueued on its stream and reports a device-side
+ * bounded-wait expiry of an earlier asynchronous call as FD_ERR_TIMEOUT (the status is cleared
+ * once reported). */
+fd_status fd_synchronize(fd_ctx* ctx);
 
 /* The single primitive of Sec. 2.1 with both diagonal scalings explicit:
  *   Y = diag(left) K(Xrow, X) diag(right) V,  K_ij = exp(-beta |xrow_i - x_j|^2).

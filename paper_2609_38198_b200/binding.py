@@ -25,7 +25,7 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 # Every symbol include/fd.h declares (checked by the CPU test-suite against the header).
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
-    "fd_apply", "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree",
+    "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree",
     "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
@@ -61,6 +61,7 @@ def _load() -> ctypes.CDLL:
     lib.fd_beta0.argtypes = [c_void_p, POINTER(c_double)]
     lib.fd_degree.argtypes = [c_void_p, c_double, c_double, c_int32, c_void_p, c_void_p, c_void_p,
                               POINTER(c_double), POINTER(c_double)]
+    lib.fd_synchronize.argtypes = [c_void_p]
     lib.fd_apply.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_void_p, c_int64, c_int32]
     lib.fd_apply_general.argtypes = [c_void_p, c_double, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_void_p,
                                      c_int64, c_int32, c_void_p, c_int64, c_int32]
@@ -72,7 +73,7 @@ def _load() -> ctypes.CDLL:
     lib.fd_nystrom.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int32, POINTER(c_double),
                                c_void_p, c_int64]
     lib.fd_scale_by_degree.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_double, c_void_p, c_int64]
-    for name in ("fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree", "fd_apply",
+    for name in ("fd_synchronize", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree", "fd_apply",
                  "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree"):
         getattr(lib, name).restype = c_int32
     lib.fd_status_string.argtypes = [c_int32]
@@ -182,6 +183,10 @@ class Context:
         with torch.cuda.device(self.device):
             self._check(lib.fd_degree(self._h, beta, alpha, prec, _ptr(q), _ptr(d), _ptr(s), byref(so), byref(so2)))
         return q, d, s, so.value, so2.value
+
+    def synchronize(self):
+        with torch.cuda.device(self.device):
+            self._check(lib.fd_synchronize(self._h))
 
     def apply(self, V: torch.Tensor, out: torch.Tensor | None = None, prec: int = FD_PREC_FP32) -> torch.Tensor:
         if V.dim() == 1:

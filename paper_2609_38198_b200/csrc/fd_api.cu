@@ -120,6 +120,8 @@ fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int6
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
     if (e != cudaSuccess) { delete c; return FD_ERR_CUDA; }
+    e = cudaMemsetAsync(c->at<unsigned int>(L.status), 0, 256, c->stream);
+    if (e != cudaSuccess) { delete c; return FD_ERR_CUDA; }
     fd_status st = setup_points(c, X_dev, ldx);
     if (st != FD_OK) { delete c; return st; }
     *out = c;
@@ -142,6 +144,9 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "flush")) {
         if (v < 0 || v > 1 << 20) return fail(c, FD_ERR_INVALID, "flush out of range");
         c->opt_flush = (int)v;
+    } else if (!strcmp(name, "tc_max_mag")) {
+        if (!(v > 0)) return fail(c, FD_ERR_INVALID, "tc_max_mag must be positive");
+        c->opt_tc_max_mag = v;
     } else if (!strcmp(name, "poly_exp")) {
         if (v < 0 || v > 1) return fail(c, FD_ERR_INVALID, "poly_exp out of range");
         c->opt_poly = v;
@@ -157,6 +162,7 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "splits")) *v = c->opt_splits;
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "poly_exp")) *v = c->opt_poly;
+    else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "mean_sq")) *v = c->mean_sq;
     else if (!strcmp(name, "max_sq")) *v = c->max_sq;
     else if (!strcmp(name, "beta")) *v = c->beta;
@@ -196,14 +202,14 @@ fd_status fd_degree(fd_ctx* c, double beta, double alpha, fd_precision prec, flo
         // pass 2: d = q^-alpha * K q^-alpha
         FD_TRY(ew_pow(c, c->q(), -alpha, c->w(), N));
         ApplyArgs a2 = a;
-        a2.left = c->w(); a2.right = c->w(); a2.Y = c->d(); a2.rowsq = nullptr;
+        a2.left = c->w(); a2.right = c->w(); a2.Y = c->d(); a2.rowsq = nullptr; a2.right_pos = true;
         FD_TRY(apply_dispatch(c, a2));
         FD_TRY(ew_scale_vec(c, c->w(), c->d(), c->s(), N));
     }
     if (q_dev) FD_CUDA(c, cudaMemcpyAsync(q_dev, c->q(), (size_t)N * 4, cudaMemcpyDeviceToDevice, c->stream));
     if (d_dev) FD_CUDA(c, cudaMemcpyAsync(d_dev, c->d(), (size_t)N * 4, cudaMemcpyDeviceToDevice, c->stream));
     if (s_dev) FD_CUDA(c, cudaMemcpyAsync(s_dev, c->s(), (size_t)N * 4, cudaMemcpyDeviceToDevice, c->stream));
-    FD_CUDA(c, cudaStreamSynchronize(c->stream));
+    FD_TRY(tc_check_status(c));
     // the diagonal of K is exactly 1 in both sums
     if (S_off_host) *S_off_host = sum_q - (double)N;
     if (S_off_2beta_host) *S_off_2beta_host = sum_sq - (double)N;
@@ -269,6 +275,11 @@ fd_status fd_scale_by_degree(fd_ctx* c, const float* v_dev, int64_t ldv, int32_t
     FD_TRY(check_block(c, v_dev, ldv, c->L.N, "v"));
     FD_TRY(check_block(c, out_dev, ldout, c->L.N, "out"));
     return scale_cols_by_pow(c, v_dev, ldv, cols, c->d(), power, out_dev, ldout, c->L.N);
+}
+
+fd_status fd_synchronize(fd_ctx* c) {
+    if (!c) return FD_ERR_INVALID;
+    return tc_check_status(c);
 }
 
 const char* fd_status_string(fd_status st) {

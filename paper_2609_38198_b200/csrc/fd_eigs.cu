@@ -62,7 +62,7 @@ struct Solver {
             FD_TRY(fd_apply(c, Q + (int64_t)(c0 + o) * N, N, w, W + (int64_t)(c0 + o) * N, N, FD_PREC_FP32));
             ++applies;
         }
-        FD_CUDA(c, cudaStreamSynchronize(c->stream));
+        FD_TRY(tc_check_status(c));
         t_apply += secs(t0, clk::now());
         return FD_OK;
     }

@@ -55,6 +55,7 @@ struct fd_ctx {
     int opt_splits = 0;
     int opt_flush = 0;
     double opt_poly = 0.0;
+    double opt_tc_max_mag = 128.0;   // largest beta' * max|x - mu|^2 the Gram-form kernel is trusted with in fp32 mode
     std::string err;
 
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -106,12 +107,15 @@ struct ApplyArgs {
     const float* V; int64_t ldv; int32_t b;
     float* Y; int64_t ldy;
     double* rowsq;                          // optional: sum_j K_ij^2 per row (rowsum mode, b = 1, V null)
+    bool right_pos;                         // caller guarantees right > 0 elementwise
     fd_precision prec;
 };
 fd_status apply_simt(fd_ctx* c, const ApplyArgs& a);
 fd_status apply_tc(fd_ctx* c, const ApplyArgs& a);
 bool tc_supported(const fd_ctx* c, const ApplyArgs& a);
 fd_status apply_dispatch(fd_ctx* c, const ApplyArgs& a);
+// Reads and clears the tensor-core kernel's status word; FD_ERR_TIMEOUT if a bounded wait expired.  Synchronises.
+fd_status tc_check_status(fd_ctx* c);
 
 // ---- small kernels (fd_elementwise.cu) ------------------------------------------------------
 fd_status ew_pow(fd_ctx* c, const float* in, double p, float* out, int64_t n);            // out = in^p

@@ -1,13 +1,761 @@
-// Tensor-core (tcgen05 / TMEM) Gram-form kernel.  Placeholder until the kernel lands: reports
-// that no shape is covered, so every call is served by the direct-difference kernels.
+// Gram-form kernel on the 5th-generation tensor cores (tcgen05 + TMEM), Eqs. 4-6.
+//
+// Per (row tile I, column tile J) of 128 x 128 pairs:
+//   1. Gram MMA (fp16 hi/lo split, three products per 16-wide K slab, fp32 accumulation in TMEM)
+//      of AUGMENTED points, so the tile leaves the tensor core already as the base-2 exponent
+//        S_ij = 2 b' x_i.x_j - b' r_i - b' r_j + bias            (b' = beta log2 e, Eq. 4)
+//      the norms ride along as extra K columns ([.., e_i, 1] . [.., 1, e_j]), each norm carried by
+//      two hi/lo pairs so it is exact to fp32.
+//   2. Two warpgroups (one per row tile; thread = row) read S from TMEM, take 2^S on the MUFU,
+//      split P = 2^S into fp16 hi + lo (mask / subtract), and write both halves back IN PLACE over
+//      the S columns as the TMEM A operand.
+//   3. Product MMA  Y_I += P_hi W_hi + P_lo W_hi + P_hi W_lo  with W = diag(right) V pre-split into
+//      fp16 hi / lo (per-column power-of-two scaling), fp32 accumulation in TMEM (Eq. 6).
+//   4. Every `flush` column tiles the TMEM accumulator is added into fp32 registers and restarted,
+//      so tensor-core accumulation error does not grow with N (two TMEM accumulators per row
+//      tile alternate, so the MMA never waits for the flush).
+// Row-sum mode (degree passes): no product MMA; the warpgroups add P (and P^2) on the FMA pipe,
+// fp32 within a column tile and fp64 across tiles; a positive right vector enters through e_j.
+//
+// One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 / 6-9 = the two
+// exponential warpgroups.  Column tiles are staged by TMA (no multicast) through a 4-deep ring.
+// Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains and exits.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cmath>
+
 #include "fd_internal.h"
 
 namespace fd {
 
-bool tc_supported(const fd_ctx*, const ApplyArgs&) { return false; }
+namespace {
 
-fd_status apply_tc(fd_ctx* c, const ApplyArgs&) {
-    return fail(c, FD_ERR_UNSUPPORTED, "tensor-core path not built");
+constexpr int kStages = 4;
+constexpr int kThreads = 320;
+constexpr int kBias = 15;                    // P' = 2^15 P keeps fp16 hi/lo of P out of the denormal range
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any legitimate wait
+
+enum Mode { kModeBlock = 0, kModeFast = 1, kModeRowsum = 2 };
+
+struct TcParams {
+    int64_t Nrow, N;             // valid rows / columns
+    int num_work;                // row-pair tiles (256 rows each)
+    int num_jt;                  // column tiles
+    int64_t np_rows;             // padded row count of the operand arrays (row index of K slab c = c * np + p)
+    int64_t np_cols;
+    int K16;
+    int b;                       // real block columns to store
+    int flush;                   // column tiles per accumulator flush
+    const float* left;           // may be null
+    const float* colscale_inv;   // per column: 2^-bias / colscale
+    float* Y; int64_t ldy;
+    float* q; double* rowsq;     // row-sum outputs
+    unsigned int* status;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: returns false (and raises the abort flag) when the limit is hit or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                atomicCAS(status, 0u, (unsigned)(0x100 | code));
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// K-major shared-memory operand descriptor (sm_100 format): start address, stride between 8-row groups,
+// swizzle mode (2 = 128 B rows, 4 = 64 B rows).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)(sbo_bytes >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)layout << 61;
+    return d;
+}
+// Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t idesc_f16(int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------ shared memory map
+template <int BT, int MODE>
+struct Smem {
+    static constexpr int kXChunk = 128 * 64;                       // one K slab (hi|lo) of 128 points: 8 KB
+    static constexpr int kWHalf = (MODE == kModeRowsum) ? 0 : BT * 128;   // 64 j x BT columns fp16
+    static constexpr int kWBytes = (MODE == kModeRowsum) ? 0 : (MODE == kModeFast ? 2 : 4) * kWHalf;
+    static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
+    static __host__ __device__ constexpr int total(int K16) {
+        return 1024 /*align slack*/ + kStages * stage_bytes(K16) + 2 * K16 * kXChunk + 1024 /*barriers*/;
+    }
+};
+
+struct Barriers {
+    uint64_t full[kStages], empty[kStages];
+    uint64_t xfull, xempty;
+    uint64_t s_full[2], p_full[2];          // block mode: S ready / P written (per row tile)
+    uint64_t s_free[2][2];                  // row-sum mode: S buffer consumed (per row tile, per buffer)
+    uint64_t s_full2[2][2];                 // row-sum mode: S buffer ready
+    uint64_t y_full[2][2], y_empty[2][2];   // accumulator flush hand-off (per row tile, per buffer)
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// ------------------------------------------------------------------------------------------------ the kernel
+template <int BT, int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUtensorMap map_xcol,
+     const __grid_constant__ CUtensorMap map_whi, const __grid_constant__ CUtensorMap map_wlo, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    using SM = Smem<BT, MODE>;
+    const int K16 = p.K16;
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_base = base;
+    uint8_t* xi_base = base + kStages * SM::stage_bytes(K16);                 // 2 row tiles x K16 slabs
+    Barriers* bars = (Barriers*)(xi_base + 2 * K16 * SM::kXChunk);
+    volatile int* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&bars->s_full[t], 1); mbar_init(&bars->p_full[t], 4);
+            for (int u = 0; u < 2; ++u) {
+                mbar_init(&bars->s_free[t][u], 4); mbar_init(&bars->s_full2[t][u], 1);
+                mbar_init(&bars->y_full[t][u], 1); mbar_init(&bars->y_empty[t][u], 4);
+            }
+        }
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    const int num_jt = p.num_jt;
+    const int my_items = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int flush = p.flush;
+
+    // TMEM columns: row tile t owns [256 t, 256 t + 256): S (or S buffer 0) at +0, block mode: Y buffers at +128, +192;
+    // row-sum mode: S buffer 1 at +128.
+    if (warp == 0) {
+        // =============================================================== TMA producer (one thread)
+        if (lane == 0) {
+            prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol);
+            if (MODE != kModeRowsum) { prefetch_tmap(&map_whi); if (MODE == kModeBlock) prefetch_tmap(&map_wlo); }
+            uint32_t it = 0;
+            bool ok = true;
+            for (int w = 0; w < my_items && ok; ++w) {
+                const int item = blockIdx.x + w * gridDim.x;
+                ok = mbar_wait(&bars->xempty, (w & 1) ^ 1, abort_flag, p.status, 1);
+                if (!ok) break;
+                mbar_expect_tx(&bars->xfull, 2 * K16 * SM::kXChunk);
+                for (int t = 0; t < 2; ++t)
+                    for (int c = 0; c < K16; ++c)
+                        tma_load_2d(xi_base + (t * K16 + c) * SM::kXChunk, &map_xrow, 0,
+                                    (int)(c * p.np_rows + (int64_t)item * 256 + t * 128), &bars->xfull);
+                for (int j = 0; j < num_jt; ++j, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(&bars->empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.status, 2);
+                    if (!ok) break;
+                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                    mbar_expect_tx(&bars->full[s], SM::stage_bytes(K16));
+                    for (int c = 0; c < K16; ++c)
+                        tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)j * 128), &bars->full[s]);
+                    if (MODE != kModeRowsum) {
+                        uint8_t* wst = st + K16 * SM::kXChunk;
+                        tma_load_2d(wst, &map_whi, j * 128, 0, &bars->full[s]);
+                        tma_load_2d(wst + SM::kWHalf, &map_whi, j * 128 + 64, 0, &bars->full[s]);
+                        if (MODE == kModeBlock) {
+                            tma_load_2d(wst + 2 * SM::kWHalf, &map_wlo, j * 128, 0, &bars->full[s]);
+                            tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, j * 128 + 64, 0, &bars->full[s]);
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // aborted: let the copies already in flight land before the CTA exits (bounded)
+                const uint32_t issued = it;
+                for (uint32_t k = (issued > (uint32_t)kStages ? issued - kStages : 0); k < issued; ++k) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&bars->full[k % kStages], (k / kStages) & 1) && clock64() - t0 < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =============================================================== MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc_g = idesc_f16(128);
+            constexpr uint32_t idesc_y = idesc_f16(BT);
+            uint32_t it = 0;                 // column-tile counter across work items (stage ring)
+            uint32_t n_s[2] = {0, 0};        // S tiles produced per row tile
+            uint32_t n_p[2] = {0, 0};        // P tiles consumed per row tile
+            uint32_t n_grp[2] = {0, 0};      // accumulator groups started per row tile
+            bool ok = true;
+
+            auto gram = [&](int t, int s, uint32_t s_col) {
+                uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                for (int c = 0; c < K16; ++c) {
+                    const uint32_t a = smem_u32(xi_base + (t * K16 + c) * SM::kXChunk);
+                    const uint32_t b = smem_u32(st + c * SM::kXChunk);
+                    const uint64_t a_hi = smem_desc(a, 512, 4), a_lo = smem_desc(a + 32, 512, 4);
+                    const uint64_t b_hi = smem_desc(b, 512, 4), b_lo = smem_desc(b + 32, 512, 4);
+                    mma_ss(tmem + s_col, a_hi, b_hi, idesc_g, c > 0);
+                    mma_ss(tmem + s_col, a_hi, b_lo, idesc_g, 1);
+                    mma_ss(tmem + s_col, a_lo, b_hi, idesc_g, 1);
+                }
+            };
+
+            for (int w = 0; w < my_items && ok; ++w) {
+                ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
+                if (!ok) break;
+                tc_fence_after();
+                if (MODE == kModeRowsum) {
+                    // S double-buffered per row tile; the warpgroups free a buffer after reading it
+                    for (int j = 0; j < num_jt && ok; ++j, ++it) {
+                        const int s = it % kStages;
+                        ok = mbar_wait(&bars->full[s], (it / kStages) & 1, abort_flag, p.status, 4);
+                        if (!ok) break;
+                        tc_fence_after();
+                        for (int t = 0; t < 2 && ok; ++t) {
+                            const uint32_t n = n_s[t]++;
+                            const int buf = n & 1;
+                            ok = mbar_wait(&bars->s_free[t][buf], ((n >> 1) & 1) ^ 1, abort_flag, p.status, 5);
+                            if (!ok) break;
+                            tc_fence_after();
+                            gram(t, s, 256 * t + 128 * buf);
+                            tc_commit(&bars->s_full2[t][buf]);
+                        }
+                        tc_commit(&bars->empty[s]);
+                    }
+                } else {
+                    // prologue: S(t, 0)
+                    ok = mbar_wait(&bars->full[it % kStages], (it / kStages) & 1, abort_flag, p.status, 4);
+                    if (!ok) break;
+                    tc_fence_after();
+                    for (int t = 0; t < 2; ++t) { gram(t, it % kStages, 256 * t); tc_commit(&bars->s_full[t]); ++n_s[t]; }
+                    for (int j = 0; j < num_jt && ok; ++j, ++it) {
+                        const int s = it % kStages;
+                        const bool has_next = j + 1 < num_jt;
+                        if (has_next) {
+                            ok = mbar_wait(&bars->full[(it + 1) % kStages], ((it + 1) / kStages) & 1, abort_flag, p.status, 4);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        const bool group_start = (j % flush) == 0;
+                        const bool group_end = ((j + 1) % flush) == 0 || !has_next;
+                        for (int t = 0; t < 2 && ok; ++t) {
+                            const int yb = n_grp[t] & 1;
+                            if (group_start) {
+                                ok = mbar_wait(&bars->y_empty[t][yb], ((n_grp[t] >> 1) & 1) ^ 1, abort_flag, p.status, 6);
+                                if (!ok) break;
+                            }
+                            ok = mbar_wait(&bars->p_full[t], n_p[t] & 1, abort_flag, p.status, 7);
+                            if (!ok) break;
+                            ++n_p[t];
+                            tc_fence_after();
+                            // Y_t += P W : 8 K steps of 16 columns j; P_hi / P_lo interleaved in 32-column chunks
+                            uint8_t* wst = stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk;
+                            const uint32_t y_col = 256 * t + 128 + 64 * yb;
+                            for (int ks = 0; ks < 8; ++ks) {
+                                const uint32_t half = ks >> 2, sub = ks & 3;
+                                const uint32_t bh = smem_u32(wst + half * SM::kWHalf) + sub * 32;
+                                const uint64_t b_hi = smem_desc(bh, 1024, 2);
+                                const uint32_t chunk = ks >> 1, h = ks & 1;
+                                const uint32_t a_hi = tmem + 256 * t + 32 * chunk + 8 * h;
+                                const uint32_t a_lo = a_hi + 16;
+                                mma_ts(tmem + y_col, a_hi, b_hi, idesc_y, !(group_start && ks == 0));
+                                if (MODE == kModeBlock) {
+                                    const uint32_t bl = smem_u32(wst + (2 + half) * SM::kWHalf) + sub * 32;
+                                    const uint64_t b_lo = smem_desc(bl, 1024, 2);
+                                    mma_ts(tmem + y_col, a_lo, b_hi, idesc_y, 1);
+                                    mma_ts(tmem + y_col, a_hi, b_lo, idesc_y, 1);
+                                }
+                            }
+                            if (group_end) { tc_commit(&bars->y_full[t][yb]); ++n_grp[t]; }
+                            if (t == 1) tc_commit(&bars->empty[s]);
+                            if (has_next) { gram(t, (it + 1) % kStages, 256 * t); tc_commit(&bars->s_full[t]); ++n_s[t]; }
+                        }
+                    }
+                }
+                if (ok) tc_commit(&bars->xempty);
+            }
+        }
+    } else {
+        // =============================================================== exponential warpgroups
+        const int t = (warp - 2) >> 2;                 // row tile of this warpgroup
+        const int wq = warp & 3;                       // TMEM lane quarter this warp may access
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        const int row_in_tile = wq * 32 + lane;
+        uint32_t n_s = 0, n_grp = 0;
+        bool ok = true;
+
+        for (int w = 0; w < my_items && ok; ++w) {
+            const int item = blockIdx.x + w * gridDim.x;
+            const int64_t row = (int64_t)item * 256 + t * 128 + row_in_tile;
+            if (MODE == kModeRowsum) {
+                double dsum = 0.0, dsq = 0.0;
+                for (int j = 0; j < num_jt && ok; ++j) {
+                    const uint32_t n = n_s++;
+                    const int buf = n & 1;
+                    ok = mbar_wait(&bars->s_full2[t][buf], (n >> 1) & 1, abort_flag, p.status, 8);
+                    if (!ok) break;
+                    tc_fence_after();
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, q0 = 0.f, q1 = 0.f;
+#pragma unroll 1
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem + lane_addr + 256 * t + 128 * buf + 32 * ch, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const float p0 = ex2f(__uint_as_float(v[i])), p1 = ex2f(__uint_as_float(v[i + 1]));
+                            const float p2 = ex2f(__uint_as_float(v[i + 2])), p3 = ex2f(__uint_as_float(v[i + 3]));
+                            a0 += p0; a1 += p1; a2 += p2; a3 += p3;
+                            q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1); q0 = fmaf(p2, p2, q0); q1 = fmaf(p3, p3, q1);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->s_free[t][buf]);
+                    dsum += (double)((a0 + a1) + (a2 + a3));
+                    dsq += (double)(q0 + q1);
+                }
+                if (ok && row < p.Nrow) {
+                    const double l = p.left ? (double)p.left[row] : 1.0;
+                    p.q[row] = (float)(dsum * l);
+                    if (p.rowsq) p.rowsq[row] = dsq;
+                }
+            } else {
+                float acc[BT];
+#pragma unroll
+                for (int c = 0; c < BT; ++c) acc[c] = 0.f;
+                for (int j = 0; j < num_jt && ok; ++j) {
+                    ok = mbar_wait(&bars->s_full[t], n_s & 1, abort_flag, p.status, 9);
+                    if (!ok) break;
+                    ++n_s;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t v[32];
+                        const uint32_t addr = tmem + lane_addr + 256 * t + 32 * ch;
+                        tmem_ld32(addr, v);
+                        tmem_wait_ld();
+                        uint32_t hi[16], lo[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float p0 = ex2f(__uint_as_float(v[2 * i])), p1 = ex2f(__uint_as_float(v[2 * i + 1]));
+                            if (MODE == kModeBlock) {
+                                const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
+                                const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
+                                hi[i] = pack_f16x2(h0, h1);
+                                lo[i] = pack_f16x2(p0 - h0, p1 - h1);
+                            } else {
+                                hi[i] = pack_f16x2(p0, p1);
+                            }
+                        }
+                        tmem_st16(addr, hi);
+                        if (MODE == kModeBlock) tmem_st16(addr + 16, lo);
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->p_full[t]);
+                    // accumulator flush: the group that ends with this column tile
+                    if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
+                        const int yb = n_grp & 1;
+                        ok = mbar_wait(&bars->y_full[t][yb], (n_grp >> 1) & 1, abort_flag, p.status, 10);
+                        if (!ok) break;
+                        ++n_grp;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c0 = 0; c0 < BT; c0 += 32) {
+                            if (BT >= 32) {
+                                uint32_t v[32];
+                                tmem_ld32(tmem + lane_addr + 256 * t + 128 + 64 * yb + c0, v);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) acc[c0 + i] += __uint_as_float(v[i]);
+                            }
+                        }
+                        if (BT == 16) {
+                            uint32_t v[32];
+                            // a 16-column accumulator is read with one 32-column load; the upper half is ignored
+                            tmem_ld32(tmem + lane_addr + 256 * t + 128 + 64 * yb, v);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) acc[i] += __uint_as_float(v[i]);
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->y_empty[t][yb]);
+                    }
+                }
+                if (ok && row < p.Nrow) {
+                    const float l = p.left ? p.left[row] : 1.0f;
+#pragma unroll
+                    for (int c = 0; c < BT; ++c)
+                        if (c < p.b) p.Y[row + (int64_t)c * p.ldy] = acc[c] * l * p.colscale_inv[c];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ operand packing
+// Augmented fp16 hi|lo operand rows.  role 0 (rows of the product): [c x, e, 1]; role 1 (columns): [c x, 1, e] with
+// c = sqrt(2 b'), e = -b' |x - mu|^2 (+ extra_j: bias and log2 of a positive right vector for role 1).
+// Layout: slab s (16 augmented columns) of point p at out[(s * np + p) * 32 ..]: 16 hi then 16 lo halves.
+__global__ void k_pack_points(const float* __restrict__ xs, int DP, int D, int64_t n, int64_t np, const double* __restrict__ mu,
+                              double bprime, int role, double bias, const float* __restrict__ logw_src, int K16,
+                              __half* __restrict__ out) {
+    int64_t pidx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pidx >= np) return;
+    const bool valid = pidx < n;
+    const double cs = sqrt(2.0 * bprime);
+    double r = 0.0;
+    if (valid)
+        for (int k = 0; k < D; ++k) { double v = (double)xs[pidx * DP + k] - mu[k]; r += v * v; }
+    double e = -bprime * r;
+    if (role == 1) {
+        e += bias;
+        if (logw_src && valid) e += log2((double)logw_src[pidx]);
+        if (!valid) e = -30000.0;                       // padded column: 2^e = 0
+    }
+    // norm pieces: two hi/lo pairs carry e to beyond fp32 precision
+    const __half e_h1 = __double2half(e);
+    const double r1 = e - (double)__half2float(e_h1);
+    const __half e_l1 = __double2half(r1);
+    const double r2 = r1 - (double)__half2float(e_l1);
+    const __half e_h2 = __double2half(r2);
+    const __half e_l2 = __double2half(r2 - (double)__half2float(e_h2));
+    const __half one = __float2half(1.0f), zero = __float2half(0.0f);
+    for (int s = 0; s < K16; ++s) {
+        __half* o = out + ((int64_t)s * np + pidx) * 32;
+        for (int kk = 0; kk < 16; ++kk) {
+            const int col = s * 16 + kk;
+            __half h = zero, l = zero;
+            if (col < D) {
+                if (valid) {
+                    const double v = cs * ((double)xs[pidx * DP + col] - mu[col]);
+                    h = __double2half(v);
+                    l = __double2half(v - (double)__half2float(h));
+                }
+            } else if (col == D || col == D + 1) {          // row-norm slots: role 0 carries e, role 1 carries 1
+                if (role == 0) { h = col == D ? e_h1 : e_h2; l = col == D ? e_l1 : e_l2; if (!valid) { h = zero; l = zero; } }
+                else h = one;
+            } else if (col == D + 2 || col == D + 3) {      // column-norm slots
+                if (role == 1) { h = col == D + 2 ? e_h1 : e_h2; l = col == D + 2 ? e_l1 : e_l2; }
+                else h = one;
+            }
+            o[kk] = h;
+            o[16 + kk] = l;
+        }
+    }
+}
+
+// Stage 1: per-block maxima of |right_j V_jc| for each column c.
+__global__ void k_colmax_partial(const float* __restrict__ V, int64_t ldv, const float* __restrict__ right, int64_t N, int c0,
+                                 int bc, float* __restrict__ part) {
+    __shared__ float sm[256];
+    const int c = blockIdx.y;
+    float m = 0.f;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < N; j += (int64_t)gridDim.x * blockDim.x) {
+        float v = V[j + (int64_t)(c0 + c) * ldv];
+        if (right) v *= right[j];
+        m = fmaxf(m, fabsf(v));
+    }
+    sm[threadIdx.x] = m;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+        if (threadIdx.x < off) sm[threadIdx.x] = fmaxf(sm[threadIdx.x], sm[threadIdx.x + off]);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) part[(size_t)c * gridDim.x + blockIdx.x] = sm[0];
+    (void)bc;
+}
+// Stage 2: column scale = power of two that puts the column maximum in [2^12, 2^13); stores the scale and the
+// epilogue factor 2^-bias / scale.
+__global__ void k_colscale(const float* __restrict__ part, int blocks, int bc, int BT, float* __restrict__ scale,
+                           float* __restrict__ inv) {
+    const int c = threadIdx.x;
+    if (c >= BT) return;
+    float m = 0.f;
+    if (c < bc)
+        for (int b = 0; b < blocks; ++b) m = fmaxf(m, part[(size_t)c * blocks + b]);
+    float sc = 1.0f;
+    if (m > 0.f && isfinite(m)) {
+        int e;
+        frexpf(m, &e);                               // m = f * 2^e, f in [0.5, 1)
+        sc = ldexpf(1.0f, 13 - e);
+    }
+    scale[c] = sc;
+    inv[c] = ldexpf(1.0f, -kBias) / sc;
+}
+// wt_hi / wt_lo [c * np + j] = fp16 split of scale_c * right_j * V[j, c0 + c]; zero padding for j >= N and c >= bc.
+__global__ void k_pack_wt(const float* __restrict__ V, int64_t ldv, const float* __restrict__ right, int64_t N, int64_t np,
+                          int c0, int bc, const float* __restrict__ scale, __half* __restrict__ hi, __half* __restrict__ lo) {
+    const int c = blockIdx.y;
+    const float sc = scale[c];
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < np; j += (int64_t)gridDim.x * blockDim.x) {
+        float v = 0.f;
+        if (c < bc && j < N) {
+            v = V[j + (int64_t)(c0 + c) * ldv];
+            if (right) v *= right[j];
+            v *= sc;
+        }
+        const __half h = __float2half_rn(v);
+        hi[(int64_t)c * np + j] = h;
+        if (lo) lo[(int64_t)c * np + j] = __float2half_rn(v - __half2float(h));
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes, uint32_t box_inner,
+                 uint32_t box_outer, CUtensorMapSwizzle sw) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BT, int MODE>
+fd_status launch_tc(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, const CUtensorMap& mh, const CUtensorMap& ml,
+                    const TcParams& p, int grid) {
+    const int smem = Smem<BT, MODE>::total(p.K16);
+    if (smem > 227 * 1024) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core kernel needs %d B of shared memory", smem);
+    static bool configured = false;
+    if (!configured) {
+        FD_CUDA(c, cudaFuncSetAttribute(k_tc<BT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        configured = true;
+    }
+    k_tc<BT, MODE><<<grid, kThreads, smem, c->stream>>>(mr, mc, mh, ml, p);
+    FD_LAUNCH_CHECK(c, "k_tc");
+    return FD_OK;
+}
+
+}  // namespace
+
+bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
+    const Layout& L = c->L;
+    if (!c->centered) return false;
+    if (L.K16 > 4) return false;                                   // D <= 60
+    if (a.Nrow > L.N) return false;
+    const double bprime = a.beta * kLog2e;
+    // exponent magnitude the fp16 hi/lo norm pieces and the fp32 Gram accumulation can carry accurately
+    const double mag = bprime * c->max_sq;
+    if (!(mag < (a.prec == FD_PREC_FAST ? 2000.0 : c->opt_tc_max_mag))) return false;
+    if (a.V == nullptr) return a.right == nullptr || a.right_pos;  // row-sum mode folds a positive right vector into e_j
+    if (c->opt_path != FD_PATH_TC && L.N < 16384) return false;    // small problems: the split direct-difference kernel fills the GPU better
+    return true;
+}
+
+fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
+    const Layout& L = c->L;
+    const int64_t N = L.N, NP = L.NP;
+    if (!encode_fn()) return fail(c, FD_ERR_CUDA, "cuTensorMapEncodeTiled entry point unavailable");
+    const double bprime = a.beta * kLog2e;
+    const bool rowsum = a.V == nullptr;
+    const double* mu = c->at<double>(L.mu);
+    __half* xp_col = c->at<__half>(L.xp_col);
+    __half* xp_row = c->at<__half>(L.xp_row);
+    unsigned int* status = c->at<unsigned int>(L.status);
+    const int K16 = L.K16;
+    const int pk_blocks = (int)ceil_div(NP, 256);
+    // operands: columns (role 1) always from the context's points, rows (role 0) from a.xrow
+    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(c->xs(), L.DP, L.D, N, NP, mu, bprime, 1, rowsum ? 0.0 : (double)kBias,
+                                                   rowsum ? a.right : nullptr, K16, xp_col);
+    FD_LAUNCH_CHECK(c, "k_pack_points(col)");
+    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(a.xrow, L.DP, L.D, a.Nrow, NP, mu, bprime, 0, 0.0, nullptr, K16, xp_row);
+    FD_LAUNCH_CHECK(c, "k_pack_points(row)");
+
+    CUtensorMap mr, mc, mh, ml;
+    if (!make_map_2d(&mr, xp_row, 32, (uint64_t)K16 * NP, 64, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map_2d(&mc, xp_col, 32, (uint64_t)K16 * NP, 64, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B))
+        return fail(c, FD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the point operands");
+
+    TcParams p{};
+    p.Nrow = a.Nrow; p.N = N;
+    p.num_work = (int)ceil_div(a.Nrow, 256);
+    p.num_jt = (int)ceil_div(N, 128);
+    p.np_rows = NP; p.np_cols = NP; p.K16 = K16;
+    p.left = a.left; p.status = status;
+    p.flush = c->opt_flush > 0 ? c->opt_flush : 4;
+    const int grid = std::min(p.num_work, c->sm_count);
+
+    if (rowsum) {
+        p.q = a.Y; p.rowsq = a.rowsq; p.b = 1;
+        FD_TRY((launch_tc<16, kModeRowsum>(c, mr, mc, mc, mc, p, grid)));
+    } else {
+        __half* wt_hi = c->at<__half>(L.wt_hi);
+        __half* wt_lo = c->at<__half>(L.wt_lo);
+        float* scale = c->at<float>(L.colscale);
+        float* inv = scale + L.BP + 8;
+        float* part = c->at<float>(L.part);
+        const bool fast = a.prec == FD_PREC_FAST;
+        for (int c0 = 0; c0 < a.b; c0 += 64) {
+            const int bc = std::min(64, a.b - c0);
+            const int BT = bc <= 16 ? 16 : bc <= 32 ? 32 : 64;
+            const int cm_blocks = (int)std::min<int64_t>(256, ceil_div(N, 1024));
+            k_colmax_partial<<<dim3(cm_blocks, bc), 256, 0, c->stream>>>(a.V, a.ldv, a.right, N, c0, bc, part);
+            FD_LAUNCH_CHECK(c, "k_colmax_partial");
+            k_colscale<<<1, 64, 0, c->stream>>>(part, cm_blocks, bc, BT, scale, inv);
+            FD_LAUNCH_CHECK(c, "k_colscale");
+            k_pack_wt<<<dim3((unsigned)std::min<int64_t>(1024, ceil_div(NP, 256)), BT), 256, 0, c->stream>>>(
+                a.V, a.ldv, a.right, N, NP, c0, bc, scale, wt_hi, fast ? nullptr : wt_lo);
+            FD_LAUNCH_CHECK(c, "k_pack_wt");
+            if (!make_map_2d(&mh, wt_hi, (uint64_t)NP, (uint64_t)BT, (uint64_t)NP * 2, 64, BT, CU_TENSOR_MAP_SWIZZLE_128B) ||
+                !make_map_2d(&ml, wt_lo, (uint64_t)NP, (uint64_t)BT, (uint64_t)NP * 2, 64, BT, CU_TENSOR_MAP_SWIZZLE_128B))
+                return fail(c, FD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the block operands");
+            p.b = bc; p.colscale_inv = inv; p.Y = a.Y + (int64_t)c0 * a.ldy; p.ldy = a.ldy;
+#define FD_TC_CASE(B)                                                                              \
+    case B:                                                                                        \
+        if (fast) FD_TRY((launch_tc<B, kModeFast>(c, mr, mc, mh, ml, p, grid)));                   \
+        else FD_TRY((launch_tc<B, kModeBlock>(c, mr, mc, mh, ml, p, grid)));                       \
+        break;
+            switch (BT) { FD_TC_CASE(16) FD_TC_CASE(32) FD_TC_CASE(64) }
+#undef FD_TC_CASE
+        }
+    }
+    return FD_OK;
+}
+
+// Reads the kernel's status word (after the stream has been synchronised by the caller).
+fd_status tc_check_status(fd_ctx* c) {
+    unsigned int h = 0;
+    FD_CUDA(c, cudaMemcpyAsync(&h, c->at<unsigned int>(c->L.status), 4, cudaMemcpyDeviceToHost, c->stream));
+    FD_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (h != 0) {
+        FD_CUDA(c, cudaMemsetAsync(c->at<unsigned int>(c->L.status), 0, 4, c->stream));
+        return fail(c, FD_ERR_TIMEOUT, "tensor-core kernel: bounded wait expired (code 0x%x)", h);
+    }
+    return FD_OK;
 }
 
 }  // namespace fd
