@@ -147,6 +147,8 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "tc_max_mag")) {
         if (!(v > 0)) return fail(c, FD_ERR_INVALID, "tc_max_mag must be positive");
         c->opt_tc_max_mag = v;
+    } else if (!strcmp(name, "trace")) {
+        c->opt_trace = (int)v;
     } else if (!strcmp(name, "poly_exp")) {
         if (v < 0 || v > 1) return fail(c, FD_ERR_INVALID, "poly_exp out of range");
         c->opt_poly = v;
@@ -163,6 +165,7 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "poly_exp")) *v = c->opt_poly;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
+    else if (!strcmp(name, "trace_offset")) *v = (double)c->L.part;
     else if (!strcmp(name, "mean_sq")) *v = c->mean_sq;
     else if (!strcmp(name, "max_sq")) *v = c->max_sq;
     else if (!strcmp(name, "beta")) *v = c->beta;

@@ -12,13 +12,16 @@
 //   3. Product MMA  Y_I += P_hi W_hi + P_lo W_hi + P_hi W_lo  with W = diag(right) V pre-split into
 //      fp16 hi / lo (per-column power-of-two scaling), fp32 accumulation in TMEM (Eq. 6).
 //   4. Every `flush` column tiles the TMEM accumulator is added into fp32 registers and restarted,
-//      so tensor-core accumulation error does not grow with N (two TMEM accumulators per row
-//      tile alternate, so the MMA never waits for the flush).
+//      so tensor-core accumulation error does not grow with N.
+// S tiles flow through a ring of TMEM buffers shared by both row tiles, so the tensor core runs ahead of
+// the warpgroups and the product MMA of a tile overlaps the exponentials of the next ones.
 // Row-sum mode (degree passes): no product MMA; the warpgroups add P (and P^2) on the FMA pipe,
 // fp32 within a column tile and fp64 across tiles; a positive right vector enters through e_j.
 //
-// One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 / 6-9 = the two
-// exponential warpgroups.  Column tiles are staged by TMA (no multicast) through a 4-deep ring.
+// One persistent CTA per SM: warps 0-3 / 4-7 = the two exponential warpgroups (raised to 232 registers);
+// warp 8 = TMA producer, warps 9 / 10 = product-MMA issuers for row tile 0 / 1, warp 11 = Gram-MMA issuer
+// (lowered to 40 registers).  Three issuing threads because the per-tile bookkeeping of a lone issuer
+// (waits, commits, descriptors) cost about as much as its MMAs and left the tensor pipe idle.  Column tiles are staged by TMA (no multicast) through a 4-deep ring.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains and exits.
 #include <cuda.h>
 
@@ -32,7 +35,7 @@ namespace fd {
 namespace {
 
 constexpr int kStages = 4;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                // warps 0-3 / 4-7: exponential warpgroups; warps 8-11: TMA, MMA, 2 idle
 constexpr int kBias = 15;                    // P' = 2^15 P keeps fp16 hi/lo of P out of the denormal range
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any legitimate wait
@@ -53,6 +56,8 @@ struct TcParams {
     float* Y; int64_t ldy;
     float* q; double* rowsq;     // row-sum outputs
     unsigned int* status;
+    int dbg;                     // tuning aid: bit 0 = warpgroups skip exponentials and stores, bit 1 = skip the S loads too
+    long long* trace;            // optional: clock64 stamps of CTA 0's first tiles (tuning aid), [4 roles][64 tiles][8 events]
 };
 
 // ------------------------------------------------------------------------------------------------ PTX
@@ -76,12 +81,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: returns false (and raises the abort flag) when the limit is hit or another role aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, int code) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(40);            // back off: many warps polling shared memory slow the MMA issuer down
         if ((++spins & 63) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycles) {
@@ -141,6 +156,19 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
         ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
           "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&v)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -170,6 +198,11 @@ __host__ __device__ constexpr uint32_t idesc_f16(int n) {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+#define FD_TRACE(role, tile, ev)                                                                   \
+    do {                                                                                          \
+        if (p.trace && blockIdx.x == 0 && (tile) < 64) p.trace[((role) * 64 + (tile)) * 8 + (ev)] = clock64(); \
+    } while (0)
+
 // ------------------------------------------------------------------------------------------------ shared memory map
 template <int BT, int MODE>
 struct Smem {
@@ -182,24 +215,32 @@ struct Smem {
     }
 };
 
+constexpr int kMaxBuf = 4;
+
 struct Barriers {
     uint64_t full[kStages], empty[kStages];
     uint64_t xfull, xempty;
-    uint64_t s_full[2], p_full[2];          // block mode: S ready / P written (per row tile)
-    uint64_t s_free[2][2];                  // row-sum mode: S buffer consumed (per row tile, per buffer)
-    uint64_t s_full2[2][2];                 // row-sum mode: S buffer ready
-    uint64_t y_full[2][2], y_empty[2][2];   // accumulator flush hand-off (per row tile, per buffer)
+    uint64_t s_full[kMaxBuf];               // S tile ready in ring buffer (MMA -> warpgroup)
+    uint64_t s_done[kMaxBuf];               // block mode: P written in place; row-sum mode: S consumed (warpgroup -> MMA)
+    uint64_t p_half[kMaxBuf];               // block mode: first 64 columns of P written (lets the product MMA start early)
+    uint64_t kw_done[kMaxBuf];              // block mode: product MMAs that read P from this buffer have completed
+    uint64_t y_full[2], y_empty[2];         // accumulator flush hand-off (per row tile)
     uint32_t tmem_base;
     int abort_flag;
 };
 
 // ------------------------------------------------------------------------------------------------ the kernel
+// Tiles of one work item are numbered n = 2 j + t (column tile j, row tile t) and flow through a ring of NBUF
+// S buffers in TMEM (3 in block mode, 4 in row-sum mode), so the tensor core runs up to NBUF tiles ahead of the
+// warpgroups and neither warpgroup waits for the product MMA of its previous tile.
 template <int BT, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUtensorMap map_xcol,
      const __grid_constant__ CUtensorMap map_whi, const __grid_constant__ CUtensorMap map_wlo, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using SM = Smem<BT, MODE>;
+    constexpr int NBUF = (MODE == kModeRowsum) ? 4 : 3;
+    constexpr uint32_t kYCol = 384;                    // block mode: Y_t at columns 384 + 64 t
     const int K16 = p.K16;
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_base = base;
@@ -210,19 +251,15 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        // a column stage is released by the Gram issuer alone (row-sum mode) or by both product issuers (block mode)
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], MODE == kModeRowsum ? 1 : 2); }
         mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(&bars->s_full[t], 1); mbar_init(&bars->p_full[t], 4);
-            for (int u = 0; u < 2; ++u) {
-                mbar_init(&bars->s_free[t][u], 4); mbar_init(&bars->s_full2[t][u], 1);
-                mbar_init(&bars->y_full[t][u], 1); mbar_init(&bars->y_empty[t][u], 4);
-            }
-        }
+        for (int u = 0; u < kMaxBuf; ++u) { mbar_init(&bars->s_full[u], 1); mbar_init(&bars->s_done[u], 4); mbar_init(&bars->kw_done[u], 1); mbar_init(&bars->p_half[u], 4); }
+        for (int t = 0; t < 2; ++t) { mbar_init(&bars->y_full[t], 1); mbar_init(&bars->y_empty[t], 4); }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -232,12 +269,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     const uint32_t tmem = bars->tmem_base;
 
     const int num_jt = p.num_jt;
+    const int tiles_per_item = 2 * num_jt;
     const int my_items = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int flush = p.flush;
 
-    // TMEM columns: row tile t owns [256 t, 256 t + 256): S (or S buffer 0) at +0, block mode: Y buffers at +128, +192;
-    // row-sum mode: S buffer 1 at +128.
-    if (warp == 0) {
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(40));
+      if (warp == 8) {
         // =============================================================== TMA producer (one thread)
         if (lane == 0) {
             prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol);
@@ -281,112 +319,124 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 }
             }
         }
-    } else if (warp == 1) {
-        // =============================================================== MMA issuer (one thread)
+      } else if (warp == 11) {
+        // =============================================================== Gram MMA issuer (one thread)
+        // Issues S(n) = A_t B_j^T for every tile as soon as its ring buffer is free again; runs up to NBUF tiles ahead.
         if (lane == 0) {
             constexpr uint32_t idesc_g = idesc_f16(128);
-            constexpr uint32_t idesc_y = idesc_f16(BT);
-            uint32_t it = 0;                 // column-tile counter across work items (stage ring)
-            uint32_t n_s[2] = {0, 0};        // S tiles produced per row tile
-            uint32_t n_p[2] = {0, 0};        // P tiles consumed per row tile
-            uint32_t n_grp[2] = {0, 0};      // accumulator groups started per row tile
+            uint32_t it0 = 0, gn0 = 0;
             bool ok = true;
-
-            auto gram = [&](int t, int s, uint32_t s_col) {
-                uint8_t* st = stage_base + s * SM::stage_bytes(K16);
-                for (int c = 0; c < K16; ++c) {
-                    const uint32_t a = smem_u32(xi_base + (t * K16 + c) * SM::kXChunk);
-                    const uint32_t b = smem_u32(st + c * SM::kXChunk);
-                    const uint64_t a_hi = smem_desc(a, 512, 4), a_lo = smem_desc(a + 32, 512, 4);
-                    const uint64_t b_hi = smem_desc(b, 512, 4), b_lo = smem_desc(b + 32, 512, 4);
-                    mma_ss(tmem + s_col, a_hi, b_hi, idesc_g, c > 0);
-                    mma_ss(tmem + s_col, a_hi, b_lo, idesc_g, 1);
-                    mma_ss(tmem + s_col, a_lo, b_hi, idesc_g, 1);
-                }
-            };
-
+            uint64_t* free_bar = (MODE == kModeRowsum) ? bars->s_done : bars->kw_done;
             for (int w = 0; w < my_items && ok; ++w) {
                 ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
                 if (!ok) break;
                 tc_fence_after();
-                if (MODE == kModeRowsum) {
-                    // S double-buffered per row tile; the warpgroups free a buffer after reading it
-                    for (int j = 0; j < num_jt && ok; ++j, ++it) {
-                        const int s = it % kStages;
-                        ok = mbar_wait(&bars->full[s], (it / kStages) & 1, abort_flag, p.status, 4);
-                        if (!ok) break;
-                        tc_fence_after();
-                        for (int t = 0; t < 2 && ok; ++t) {
-                            const uint32_t n = n_s[t]++;
-                            const int buf = n & 1;
-                            ok = mbar_wait(&bars->s_free[t][buf], ((n >> 1) & 1) ^ 1, abort_flag, p.status, 5);
-                            if (!ok) break;
-                            tc_fence_after();
-                            gram(t, s, 256 * t + 128 * buf);
-                            tc_commit(&bars->s_full2[t][buf]);
-                        }
-                        tc_commit(&bars->empty[s]);
-                    }
-                } else {
-                    // prologue: S(t, 0)
-                    ok = mbar_wait(&bars->full[it % kStages], (it / kStages) & 1, abort_flag, p.status, 4);
+                for (int n = 0; n < tiles_per_item && ok; ++n) {
+                    const uint32_t g = gn0 + (uint32_t)n;
+                    const int buf = g % NBUF;
+                    const uint32_t itj = it0 + (uint32_t)(n >> 1);
+                    const int s = itj % kStages;
+                    if (w == 0) FD_TRACE(3, n, 0);
+                    ok = mbar_wait(&free_bar[buf], ((g / NBUF) & 1) ^ 1, abort_flag, p.status, 5);
                     if (!ok) break;
-                    tc_fence_after();
-                    for (int t = 0; t < 2; ++t) { gram(t, it % kStages, 256 * t); tc_commit(&bars->s_full[t]); ++n_s[t]; }
-                    for (int j = 0; j < num_jt && ok; ++j, ++it) {
-                        const int s = it % kStages;
-                        const bool has_next = j + 1 < num_jt;
-                        if (has_next) {
-                            ok = mbar_wait(&bars->full[(it + 1) % kStages], ((it + 1) / kStages) & 1, abort_flag, p.status, 4);
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
-                        const bool group_start = (j % flush) == 0;
-                        const bool group_end = ((j + 1) % flush) == 0 || !has_next;
-                        for (int t = 0; t < 2 && ok; ++t) {
-                            const int yb = n_grp[t] & 1;
-                            if (group_start) {
-                                ok = mbar_wait(&bars->y_empty[t][yb], ((n_grp[t] >> 1) & 1) ^ 1, abort_flag, p.status, 6);
-                                if (!ok) break;
-                            }
-                            ok = mbar_wait(&bars->p_full[t], n_p[t] & 1, abort_flag, p.status, 7);
-                            if (!ok) break;
-                            ++n_p[t];
-                            tc_fence_after();
-                            // Y_t += P W : 8 K steps of 16 columns j; P_hi / P_lo interleaved in 32-column chunks
-                            uint8_t* wst = stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk;
-                            const uint32_t y_col = 256 * t + 128 + 64 * yb;
-                            for (int ks = 0; ks < 8; ++ks) {
-                                const uint32_t half = ks >> 2, sub = ks & 3;
-                                const uint32_t bh = smem_u32(wst + half * SM::kWHalf) + sub * 32;
-                                const uint64_t b_hi = smem_desc(bh, 1024, 2);
-                                const uint32_t chunk = ks >> 1, h = ks & 1;
-                                const uint32_t a_hi = tmem + 256 * t + 32 * chunk + 8 * h;
-                                const uint32_t a_lo = a_hi + 16;
-                                mma_ts(tmem + y_col, a_hi, b_hi, idesc_y, !(group_start && ks == 0));
-                                if (MODE == kModeBlock) {
-                                    const uint32_t bl = smem_u32(wst + (2 + half) * SM::kWHalf) + sub * 32;
-                                    const uint64_t b_lo = smem_desc(bl, 1024, 2);
-                                    mma_ts(tmem + y_col, a_lo, b_hi, idesc_y, 1);
-                                    mma_ts(tmem + y_col, a_hi, b_lo, idesc_y, 1);
-                                }
-                            }
-                            if (group_end) { tc_commit(&bars->y_full[t][yb]); ++n_grp[t]; }
-                            if (t == 1) tc_commit(&bars->empty[s]);
-                            if (has_next) { gram(t, (it + 1) % kStages, 256 * t); tc_commit(&bars->s_full[t]); ++n_s[t]; }
-                        }
+                    if (w == 0) FD_TRACE(3, n, 1);
+                    if ((n & 1) == 0) {
+                        ok = mbar_wait(&bars->full[s], (itj / kStages) & 1, abort_flag, p.status, 4);
+                        if (!ok) break;
                     }
+                    tc_fence_after();
+                    // The two small cross terms (hi x lo) go first and the large hi x hi term last: each MMA rounds its
+                    // result at the magnitude of its largest addend, so only the final one rounds at full magnitude.
+                    const uint32_t s_addr = tmem + 128u * buf;
+                    const int t = n & 1;
+                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                    for (int c = 0; c < K16; ++c) {
+                        const uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
+                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        mma_ss(s_addr, a, b + 2, idesc_g, c > 0);          // + 2: the lo half starts 32 B into the row
+                        mma_ss(s_addr, a + 2, b, idesc_g, 1);
+                    }
+                    for (int c = 0; c < K16; ++c) {
+                        const uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
+                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        mma_ss(s_addr, a, b, idesc_g, 1);
+                    }
+                    tc_commit(&bars->s_full[buf]);
+                    if (w == 0) FD_TRACE(3, n, 2);
+                    if (MODE == kModeRowsum && (n & 1)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
                 }
-                if (ok) tc_commit(&bars->xempty);
+                if (ok) tc_commit(&bars->xempty);                  // the row operand tiles may be replaced
+                it0 += (uint32_t)num_jt;
+                gn0 += (uint32_t)tiles_per_item;
             }
         }
+      } else if (MODE != kModeRowsum) {
+        // =============================================================== product MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1
+        // Two issuing threads so that the per-tile bookkeeping of one overlaps the MMAs of the other.
+        if (lane == 0) {
+            constexpr uint32_t idesc_y = idesc_f16(BT);
+            const int t = warp - 9;
+            uint32_t it0 = 0, gn0 = 0, n_grp = 0;
+            bool ok = true;
+            const uint32_t y_addr = tmem + kYCol + 64 * t;
+            for (int w = 0; w < my_items && ok; ++w) {
+                for (int j = 0; j < num_jt && ok; ++j) {
+                    const uint32_t g = gn0 + 2u * (uint32_t)j + (uint32_t)t;
+                    const int buf = g % NBUF;
+                    const int s = (it0 + (uint32_t)j) % kStages;
+                    if (w == 0) FD_TRACE(0, 2 * j + t, 0);
+                    ok = mbar_wait(&bars->p_half[buf], (g / NBUF) & 1, abort_flag, p.status, 7);
+                    if (!ok) break;
+                    const bool group_start = (j % flush) == 0;
+                    const bool group_end = ((j + 1) % flush) == 0 || j + 1 == num_jt;
+                    if (group_start && n_grp > 0) {
+                        ok = mbar_wait(&bars->y_empty[t], (n_grp - 1) & 1, abort_flag, p.status, 6);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    if (w == 0) FD_TRACE(0, 2 * j + t, 1);
+                    // Y_t += P W : 8 K steps of 16 columns j; K step ks reads P_hi at S-buffer columns [16 ks, 16 ks + 8)
+                    // and P_lo at [16 ks + 8, 16 ks + 16) (the warpgroup wrote them in place over S).  The first four K steps
+                    // start as soon as the first half of P is written, the rest once the tile is complete.
+                    const uint32_t wst = smem_u32(stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk);
+                    const uint64_t bd_hi = smem_desc(wst, 1024, 2);
+                    const uint64_t bd_lo = smem_desc(wst + 2 * SM::kWHalf, 1024, 2);
+                    const uint32_t p_addr = tmem + 128u * buf;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        if (ks == 4) {
+                            ok = mbar_wait(&bars->s_done[buf], (g / NBUF) & 1, abort_flag, p.status, 7);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        const uint32_t off = (uint32_t)(((ks >> 2) * SM::kWHalf + (ks & 3) * 32) >> 4);
+                        const uint32_t a_hi = p_addr + 16 * ks;
+                        mma_ts(y_addr, a_hi, bd_hi + off, idesc_y, !(group_start && ks == 0));
+                        if (MODE == kModeBlock) {
+                            mma_ts(y_addr, a_hi + 8, bd_hi + off, idesc_y, 1);
+                            mma_ts(y_addr, a_hi, bd_lo + off, idesc_y, 1);
+                        }
+                    }
+                    if (!ok) break;
+                    if (w == 0) FD_TRACE(0, 2 * j + t, 2);
+                    tc_commit(&bars->kw_done[buf]);
+                    if (group_end) { tc_commit(&bars->y_full[t]); ++n_grp; }
+                    tc_commit(&bars->empty[s]);
+                    if (w == 0) FD_TRACE(0, 2 * j + t, 3);
+                }
+                it0 += (uint32_t)num_jt;
+                gn0 += (uint32_t)tiles_per_item;
+            }
+        }
+      }
     } else {
         // =============================================================== exponential warpgroups
-        const int t = (warp - 2) >> 2;                 // row tile of this warpgroup
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(232));
+        const int t = warp >> 2;                       // row tile of this warpgroup
         const int wq = warp & 3;                       // TMEM lane quarter this warp may access
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         const int row_in_tile = wq * 32 + lane;
-        uint32_t n_s = 0, n_grp = 0;
+        uint32_t gn0 = 0, n_grp = 0;
         bool ok = true;
 
         for (int w = 0; w < my_items && ok; ++w) {
@@ -395,28 +445,31 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             if (MODE == kModeRowsum) {
                 double dsum = 0.0, dsq = 0.0;
                 for (int j = 0; j < num_jt && ok; ++j) {
-                    const uint32_t n = n_s++;
-                    const int buf = n & 1;
-                    ok = mbar_wait(&bars->s_full2[t][buf], (n >> 1) & 1, abort_flag, p.status, 8);
+                    const uint32_t g = gn0 + 2u * j + t;
+                    const int buf = g % NBUF;
+                    ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 8);
                     if (!ok) break;
                     tc_fence_after();
+                    const uint32_t addr = tmem + lane_addr + 128u * buf;
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, q0 = 0.f, q1 = 0.f;
-#pragma unroll 1
+                    uint32_t sv[4][32];
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) tmem_ld32(addr + 32 * qd, sv[qd]);
+                    tmem_wait_ld();
+                    // the buffer can be refilled as soon as its values are in registers
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->s_done[buf]);
+#pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t v[32];
-                        tmem_ld32(tmem + lane_addr + 256 * t + 128 * buf + 32 * ch, v);
-                        tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) {
-                            const float p0 = ex2f(__uint_as_float(v[i])), p1 = ex2f(__uint_as_float(v[i + 1]));
-                            const float p2 = ex2f(__uint_as_float(v[i + 2])), p3 = ex2f(__uint_as_float(v[i + 3]));
+                            const float p0 = ex2f(__uint_as_float(sv[ch][i])), p1 = ex2f(__uint_as_float(sv[ch][i + 1]));
+                            const float p2 = ex2f(__uint_as_float(sv[ch][i + 2])), p3 = ex2f(__uint_as_float(sv[ch][i + 3]));
                             a0 += p0; a1 += p1; a2 += p2; a3 += p3;
                             q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1); q0 = fmaf(p2, p2, q0); q1 = fmaf(p3, p3, q1);
                         }
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->s_free[t][buf]);
                     dsum += (double)((a0 + a1) + (a2 + a3));
                     dsq += (double)(q0 + q1);
                 }
@@ -429,21 +482,51 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 float acc[BT];
 #pragma unroll
                 for (int c = 0; c < BT; ++c) acc[c] = 0.f;
-                for (int j = 0; j < num_jt && ok; ++j) {
-                    ok = mbar_wait(&bars->s_full[t], n_s & 1, abort_flag, p.status, 9);
-                    if (!ok) break;
-                    ++n_s;
+                bool pending = false;
+                // Adds the finished TMEM accumulator of this row tile into the registers and hands it back.
+                auto do_flush = [&]() -> bool {
+                    if (!mbar_wait(&bars->y_full[t], n_grp & 1, abort_flag, p.status, 10)) return false;
+                    ++n_grp;
                     tc_fence_after();
-#pragma unroll 1
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t v[32];
-                        const uint32_t addr = tmem + lane_addr + 256 * t + 32 * ch;
-                        tmem_ld32(addr, v);
-                        tmem_wait_ld();
-                        uint32_t hi[16], lo[16];
+                    const uint32_t yaddr = tmem + lane_addr + kYCol + 64 * t;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float p0 = ex2f(__uint_as_float(v[2 * i])), p1 = ex2f(__uint_as_float(v[2 * i + 1]));
+                    for (int c0 = 0; c0 < BT; c0 += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(yaddr + c0, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[(c0 + i) % BT] += __uint_as_float(v[i]);
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->y_empty[t]);
+                    return true;
+                };
+                for (int j = 0; j < num_jt && ok; ++j) {
+                    const uint32_t g = gn0 + 2u * j + t;
+                    const int buf = g % NBUF;
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 0);
+                    ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 9);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 1);
+                    const uint32_t addr = tmem + lane_addr + 128u * buf;
+                    // whole S row into registers first (the four loads overlap), then exponentials and in-place stores
+                    uint32_t sv[4][32];
+                    if (!(p.dbg & 2)) {
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) tmem_ld32(addr + 32 * qd, sv[qd]);
+                    tmem_wait_ld();
+                    }
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 2);
+                    if (!(p.dbg & 1))
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        uint32_t hi[8], lo[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float p0 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i]));
+                            const float p1 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i + 1]));
                             if (MODE == kModeBlock) {
                                 const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
                                 const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
@@ -453,42 +536,29 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                                 hi[i] = pack_f16x2(p0, p1);
                             }
                         }
-                        tmem_st16(addr, hi);
-                        if (MODE == kModeBlock) tmem_st16(addr + 16, lo);
+                        tmem_st8(addr + 16 * ch, hi);
+                        if (MODE == kModeBlock) tmem_st8(addr + 16 * ch + 8, lo);
+                        if (ch == 3) {
+                            tmem_wait_st();
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&bars->p_half[buf]);
+                        }
                     }
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 3);
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->p_full[t]);
-                    // accumulator flush: the group that ends with this column tile
+                    if (lane == 0) mbar_arrive(&bars->s_done[buf]);
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 4);
+                    // flush of the accumulator group that ended with the PREVIOUS tile of this row tile (its product
+                    // MMA has had a whole tile of time to finish); the last group of the work item is flushed at once
+                    if (pending) { ok = do_flush(); pending = false; if (!ok) break; }
                     if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
-                        const int yb = n_grp & 1;
-                        ok = mbar_wait(&bars->y_full[t][yb], (n_grp >> 1) & 1, abort_flag, p.status, 10);
-                        if (!ok) break;
-                        ++n_grp;
-                        tc_fence_after();
-#pragma unroll
-                        for (int c0 = 0; c0 < BT; c0 += 32) {
-                            if (BT >= 32) {
-                                uint32_t v[32];
-                                tmem_ld32(tmem + lane_addr + 256 * t + 128 + 64 * yb + c0, v);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) acc[c0 + i] += __uint_as_float(v[i]);
-                            }
-                        }
-                        if (BT == 16) {
-                            uint32_t v[32];
-                            // a 16-column accumulator is read with one 32-column load; the upper half is ignored
-                            tmem_ld32(tmem + lane_addr + 256 * t + 128 + 64 * yb, v);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) acc[i] += __uint_as_float(v[i]);
-                        }
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&bars->y_empty[t][yb]);
+                        if (j + 1 == num_jt) { ok = do_flush(); if (!ok) break; }
+                        else pending = true;
                     }
+                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 5);
                 }
                 if (ok && row < p.Nrow) {
                     const float l = p.left ? p.left[row] : 1.0f;
@@ -497,11 +567,12 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         if (c < p.b) p.Y[row + (int64_t)c * p.ldy] = acc[c] * l * p.colscale_inv[c];
                 }
             }
+            gn0 += (uint32_t)tiles_per_item;
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 8) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
@@ -706,6 +777,8 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.num_jt = (int)ceil_div(N, 128);
     p.np_rows = NP; p.np_cols = NP; p.K16 = K16;
     p.left = a.left; p.status = status;
+    p.dbg = c->opt_trace >> 1;
+    p.trace = (c->opt_trace & 1) ? reinterpret_cast<long long*>(c->at<char>(L.part)) : nullptr;   // tuning aid: stamps land in the split-partials scratch
     p.flush = c->opt_flush > 0 ? c->opt_flush : 4;
     const int grid = std::min(p.num_work, c->sm_count);
 
