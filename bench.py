@@ -262,7 +262,7 @@ def run_gpu(args):
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        path_used = "simt" if ctx.get_option("path") == 1 or not TC_BUILT(fd, ctx) else "tc"
+        path_used = "tc" if ctx.get_option("last_path") == 2 else "simt"
         pairs_per_s = float(N) * N / (app_ms * 1e-3)
         mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
         mufu_peak = SM_COUNT * MUFU_PER_CLK_SM * peaks.get("sm_max_mhz", 1965.0) * 1e6       # exp / s
@@ -295,14 +295,6 @@ def run_gpu(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
-
-
-def TC_BUILT(fd, ctx) -> bool:
-    """True when the tensor-core path serves this shape (probe by option)."""
-    try:
-        return bool(ctx.get_option("tc_active"))
-    except Exception:
-        return False
 
 
 def cpu_baseline(X, V, cfg):

@@ -82,7 +82,9 @@ fd_status fd_destroy(fd_ctx* ctx);
 /* Tuning / test knobs by name: "path" (FD_PATH_*), "splits" (0 = auto), "flush" (column tiles
  * between accumulator flushes of the tensor-core kernel), "tc_max_mag" (largest beta * log2(e) *
  * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "poly_exp" (share
- * of exponentials sent to the FMA pipe, 0..1).  Unknown name -> FD_ERR_INVALID. */
+ * of exponentials sent to the FMA pipe, 0..1), "trace" (tuning aid: the tensor-core kernel stamps
+ * clock values of its first tiles into scratch).  fd_get_option also reports "last_path" (the
+ * family that served the latest pass), "beta", "mean_sq", "max_sq".  Unknown name -> FD_ERR_INVALID. */
 fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
 fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);
 

@@ -84,9 +84,11 @@ fd_status apply_dispatch(fd_ctx* c, const ApplyArgs& a) {
     int path = c->opt_path;
     if (path == FD_PATH_TC) {
         if (!tc_supported(c, a)) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core path does not cover this shape");
+        c->last_path = FD_PATH_TC;
         return apply_tc(c, a);
     }
-    if (path == FD_PATH_AUTO && tc_supported(c, a)) return apply_tc(c, a);
+    if (path == FD_PATH_AUTO && tc_supported(c, a)) { c->last_path = FD_PATH_TC; return apply_tc(c, a); }
+    c->last_path = FD_PATH_SIMT;
     return apply_simt(c, a);
 }
 
@@ -165,6 +167,7 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "poly_exp")) *v = c->opt_poly;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
+    else if (!strcmp(name, "last_path")) *v = c->last_path;
     else if (!strcmp(name, "trace_offset")) *v = (double)c->L.part;
     else if (!strcmp(name, "mean_sq")) *v = c->mean_sq;
     else if (!strcmp(name, "max_sq")) *v = c->max_sq;

@@ -474,9 +474,10 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     dsq += (double)(q0 + q1);
                 }
                 if (ok && row < p.Nrow) {
-                    const double l = p.left ? (double)p.left[row] : 1.0;
+                    // undo the 2^bias scaling of P (exact powers of two)
+                    const double l = (p.left ? (double)p.left[row] : 1.0) * (1.0 / (double)(1 << kBias));
                     p.q[row] = (float)(dsum * l);
-                    if (p.rowsq) p.rowsq[row] = dsq;
+                    if (p.rowsq) p.rowsq[row] = dsq * (1.0 / ((double)(1 << kBias) * (double)(1 << kBias)));
                 }
             } else {
                 float acc[BT];
@@ -484,7 +485,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 for (int c = 0; c < BT; ++c) acc[c] = 0.f;
                 bool pending = false;
                 // Adds the finished TMEM accumulator of this row tile into the registers and hands it back.
-                auto do_flush = [&]() -> bool {
+                // The tensor core adds each K step into the TMEM accumulator with round-toward-zero.  For a sum whose partial
+                // sums keep one sign, n additions lose n / 4 ulp of the result on average (half an ulp each, at a running
+                // magnitude that averages half the final one): measured 2.85e-8 per addition against 2^-25 = 2.98e-8.  The
+                // flush adds that expected loss back (one FMA instead of one add), which removes the common scale error of
+                // M V that would otherwise shift every eigenvalue by ~7e-7 per column tile in the group.
+                auto do_flush = [&](int tiles_in_group) -> bool {
+                    const float corr = 1.0f + (float)(tiles_in_group * 8 * (MODE == kModeBlock ? 3 : 1)) * 2.98023224e-8f;
                     if (!mbar_wait(&bars->y_full[t], n_grp & 1, abort_flag, p.status, 10)) return false;
                     ++n_grp;
                     tc_fence_after();
@@ -495,7 +502,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         tmem_ld16(yaddr + c0, v);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) acc[(c0 + i) % BT] += __uint_as_float(v[i]);
+                        for (int i = 0; i < 16; ++i) acc[(c0 + i) % BT] = fmaf(__uint_as_float(v[i]), corr, acc[(c0 + i) % BT]);
                     }
                     tc_fence_before();
                     __syncwarp();
@@ -553,9 +560,9 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 4);
                     // flush of the accumulator group that ended with the PREVIOUS tile of this row tile (its product
                     // MMA has had a whole tile of time to finish); the last group of the work item is flushed at once
-                    if (pending) { ok = do_flush(); pending = false; if (!ok) break; }
+                    if (pending) { ok = do_flush(flush); pending = false; if (!ok) break; }
                     if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
-                        if (j + 1 == num_jt) { ok = do_flush(); if (!ok) break; }
+                        if (j + 1 == num_jt) { ok = do_flush(j % flush + 1); if (!ok) break; }
                         else pending = true;
                     }
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 5);
@@ -738,12 +745,15 @@ bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
     if (!c->centered) return false;
     if (L.K16 > 4) return false;                                   // D <= 60
     if (a.Nrow > L.N) return false;
+    // The decision depends only on the data set, the bandwidth and the precision mode -- never on the kind of pass --
+    // so the degree passes and the block products of one operator always run on the same kernel family (their
+    // common rounding bias then cancels in diag(s) K diag(s)).
+    if (c->opt_path != FD_PATH_TC && L.N < 16384) return false;    // small problems: the split direct-difference kernel fills the GPU better
     const double bprime = a.beta * kLog2e;
     // exponent magnitude the fp16 hi/lo norm pieces and the fp32 Gram accumulation can carry accurately
     const double mag = bprime * c->max_sq;
     if (!(mag < (a.prec == FD_PREC_FAST ? 2000.0 : c->opt_tc_max_mag))) return false;
-    if (a.V == nullptr) return a.right == nullptr || a.right_pos;  // row-sum mode folds a positive right vector into e_j
-    if (c->opt_path != FD_PATH_TC && L.N < 16384) return false;    // small problems: the split direct-difference kernel fills the GPU better
+    if (a.V == nullptr && a.right != nullptr && !a.right_pos) return false;   // row-sum mode folds a POSITIVE right vector into e_j
     return true;
 }
 
@@ -760,7 +770,9 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     const int K16 = L.K16;
     const int pk_blocks = (int)ceil_div(NP, 256);
     // operands: columns (role 1) always from the context's points, rows (role 0) from a.xrow
-    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(c->xs(), L.DP, L.D, N, NP, mu, bprime, 1, rowsum ? 0.0 : (double)kBias,
+    // the same bias in both modes: the S tiles of the degree pass and of the block product are then bit-identical, so
+    // any rounding bias of the Gram accumulation is common to q and to K and cancels in diag(s) K diag(s)
+    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(c->xs(), L.DP, L.D, N, NP, mu, bprime, 1, (double)kBias,
                                                    rowsum ? a.right : nullptr, K16, xp_col);
     FD_LAUNCH_CHECK(c, "k_pack_points(col)");
     k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(a.xrow, L.DP, L.D, a.Nrow, NP, mu, bprime, 0, 0.0, nullptr, K16, xp_row);
@@ -779,7 +791,7 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.left = a.left; p.status = status;
     p.dbg = c->opt_trace >> 1;
     p.trace = (c->opt_trace & 1) ? reinterpret_cast<long long*>(c->at<char>(L.part)) : nullptr;   // tuning aid: stamps land in the split-partials scratch
-    p.flush = c->opt_flush > 0 ? c->opt_flush : 4;
+    p.flush = c->opt_flush > 0 ? c->opt_flush : 2;
     const int grid = std::min(p.num_work, c->sm_count);
 
     if (rowsum) {

@@ -1,0 +1,224 @@
+"""GPU parity of the tensor-core (tcgen05 / TMEM, Gram-form) kernels against the float64 oracle.
+
+Same gates as the direct-difference kernels for the block product (relative Frobenius error
+<= 1e-5 in the fp32 mode, <= 3e-3 in the fast mode).  The degree vectors q, d, s carry a small
+systematic relative bias on this path (the Gram tile is accumulated inside the tensor core at the
+magnitude of beta' |x|^2 and rounded towards zero there); it is common to all entries, cancels in
+M = diag(s) K diag(s), and is gated at 2e-5 entrywise here.
+"""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import blocked, dense
+
+pytestmark = pytest.mark.gpu
+
+TOL_APPLY = 1e-5
+TOL_FAST = 3e-3
+TOL_DEG = 2e-5
+
+
+@pytest.fixture(scope="module")
+def fd():
+    import __graft_entry__ as g
+    g.build()
+    import paper_2609_38198_b200 as fd
+    assert torch.cuda.is_available()
+    return fd
+
+
+@pytest.fixture(scope="module")
+def dev():
+    return torch.device("cuda:0")
+
+
+def relF(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    return float(np.linalg.norm(a - b) / np.linalg.norm(b))
+
+
+def tc_case(fd, dev, X, beta, alpha, b, prec=0, seed=1):
+    N = X.shape[0]
+    V = workloads.block(N, b, seed=seed)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    q, d, s, so, so2 = ctx.degree(beta, alpha, prec)
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    Y = ctx.apply(fd.to_colmajor(V, dev), prec=prec)
+    ctx.synchronize()
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    qo, do, s_o, soo, so2o = dense.degree(X, beta, alpha)
+    Yo = dense.apply(X, beta, alpha, V)
+    assert np.abs(q.cpu().numpy() / qo - 1).max() <= TOL_DEG
+    assert np.abs(d.cpu().numpy() / do - 1).max() <= 2 * TOL_DEG
+    assert np.abs(s.cpu().numpy() / s_o - 1).max() <= 2 * TOL_DEG
+    assert abs(so - soo) <= TOL_DEG * (soo + N)
+    assert abs(so2 - so2o) <= 2 * TOL_DEG * (so2o + N)
+    err = relF(Y.cpu().numpy(), Yo)
+    assert err <= (TOL_FAST if prec else TOL_APPLY), f"apply rel-Frobenius error {err:.3e}"
+    ctx.close()
+    return err
+
+
+@pytest.mark.parametrize("N", [1, 100, 256, 257, 1000, 2304])
+def test_row_and_column_tails(fd, dev, N):
+    tc_case(fd, dev, workloads.torus6(N, seed=N), 2.0, 1.0, 64 if N > 1 else 1)
+
+
+@pytest.mark.parametrize("b", [1, 8, 16, 24, 32, 64, 70, 128])
+def test_block_widths(fd, dev, b):
+    tc_case(fd, dev, workloads.torus6(900, seed=b), 1.0, 1.0, b)
+
+
+@pytest.mark.parametrize("D,beta", [(2, 3.0), (4, 3.0), (12, 2.0), (13, 1.0), (20, 1.0), (28, 0.5), (30, 1.0), (32, 0.5)])
+def test_dimensions_and_k_slabs(fd, dev, D, beta):
+    X = workloads.latent_torus(1200, seed=D, D=D) if D >= 13 else workloads.gaussian_cloud(1200, D, seed=D, scale=0.7)
+    tc_case(fd, dev, X, beta, 1.0, 32)
+
+
+@pytest.mark.parametrize("alpha", [0.0, 0.5, 1.0])
+def test_alpha(fd, dev, alpha):
+    tc_case(fd, dev, workloads.torus6(1500, seed=4), 1.5, alpha, 32)
+
+
+def test_fast_mode(fd, dev):
+    err = tc_case(fd, dev, workloads.torus6(2000, seed=5), 2.0, 1.0, 64, prec=1)
+    assert err > 1e-6            # it really is the reduced-precision path
+
+
+def test_c4_shape_reduced(fd, dev):
+    tc_case(fd, dev, workloads.latent_torus(3000), 2.0, 1.0, 32)
+
+
+@pytest.mark.parametrize("flush", [1, 2, 4, 8])
+def test_flush_interval(fd, dev, flush):
+    X = workloads.torus6(2304, seed=7)
+    V = workloads.block(2304, 64, seed=2)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=64)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    ctx.set_option("flush", flush)
+    ctx.degree(2.0, 1.0)
+    Y = ctx.apply(fd.to_colmajor(V, dev))
+    ctx.synchronize()
+    assert relF(Y.cpu().numpy(), dense.apply(X, 2.0, 1.0, V)) <= TOL_APPLY
+    ctx.close()
+
+
+def test_general_scalings_and_rectangular(fd, dev):
+    X = workloads.torus6(1100, seed=5)
+    Z = workloads.torus6(700, seed=6)
+    N = 1100
+    rng = np.random.default_rng(0)
+    l = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    r = (rng.uniform(0.5, 2.0, N) * np.where(rng.uniform(size=N) < 0.3, -1, 1)).astype(np.float32)   # signs allowed
+    lz = rng.uniform(0.5, 2.0, 700).astype(np.float32)
+    V = workloads.block(N, 16, seed=4)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=16)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    t = lambda a: torch.from_numpy(a).to(dev)
+    Vd = fd.to_colmajor(V, dev)
+    beta = 1.2
+    Y = ctx.apply_general(beta, Vd, left=t(l), right=t(r)).cpu().numpy()
+    assert relF(Y, dense.apply_general(X, beta, V, left=l, right=r)) <= TOL_APPLY
+    Y = ctx.apply_general(beta, Vd, left=t(lz), right=t(r), Xrow=t(Z)).cpu().numpy()
+    assert relF(Y, dense.apply_general(X, beta, V, left=lz, right=r, Xrow=Z)) <= TOL_APPLY
+    q1 = ctx.apply_general(beta, None).cpu().numpy()[:, 0]
+    assert np.abs(q1 / dense.degree(X, beta, 0.0)[0] - 1).max() <= TOL_DEG
+    ctx.synchronize()
+    # a zero column and a huge column in the same block (per-column scaling)
+    V2 = V.copy(); V2[:, 3] = 0.0; V2[:, 5] *= 1e6; V2[:, 7] *= 1e-6
+    Y = ctx.apply_general(beta, fd.to_colmajor(V2, dev)).cpu().numpy()
+    Yo = dense.apply_general(X, beta, V2)
+    for c in range(16):
+        if c == 3:
+            assert np.all(Y[:, c] == 0)
+        else:
+            assert relF(Y[:, c], Yo[:, c]) <= TOL_APPLY
+    ctx.close()
+
+
+def test_run_to_run_bit_reproducible(fd, dev):
+    X = workloads.torus6(3000, seed=9)
+    V = fd.to_colmajor(workloads.block(3000, 32, seed=1), dev)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=32)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    ctx.degree(1.0, 1.0)
+    a = ctx.apply(V).clone()
+    b = ctx.apply(V).clone()
+    ctx.synchronize()
+    assert torch.equal(a, b)
+    ctx.close()
+
+
+def test_eigs_on_tensor_core_path(fd, dev):
+    # same gates as the direct-difference path: eigenvalues 1e-6, residual certificate 5e-6
+    from test_gpu_eigs import check_eigs, default_m_max
+    X = workloads.torus6(3000)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=32, m_max=default_m_max(64, 32))
+    ctx.set_option("path", fd.FD_PATH_TC)
+    ctx.degree(0.5, 1.0)
+    lam, U, info = ctx.eigs(64, 32, tol=1e-6, max_applies=600)
+    check_eigs(lam, U.cpu().numpy(), X, 0.5, 1.0, 64)
+    ctx.close()
+
+
+def test_auto_path_selection(fd, dev):
+    # small problems and shapes the Gram form cannot carry accurately are served by the direct-difference kernels
+    Xs = workloads.torus6(2000, seed=1)
+    ctx = fd.Context(torch.from_numpy(Xs).to(dev), b_max=16)
+    ctx.degree(1.0, 1.0)
+    ctx.apply(fd.to_colmajor(workloads.block(2000, 16), dev))
+    assert ctx.get_option("last_path") == fd.FD_PATH_SIMT
+    ctx.close()
+    Xl = workloads.torus2(20000, seed=1)
+    ctx = fd.Context(torch.from_numpy(Xl).to(dev), b_max=16)
+    V = fd.to_colmajor(workloads.block(20000, 16), dev)
+    ctx.degree(300.0, 1.0)                 # beta' max|x|^2 = 866: beyond the Gram-form budget
+    ctx.apply(V)
+    assert ctx.get_option("last_path") == fd.FD_PATH_SIMT
+    ctx.degree(10.0, 1.0)
+    ctx.apply(V)
+    ctx.synchronize()
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    ctx.close()
+
+
+def test_full_size_sampled_rows_and_identities(fd, dev):
+    """Headline configuration (N = 2^20, D = 12, b = 64, beta = 2), the launch bench.py times: sampled rows against
+    the oracle, plus properties that hold at any size (Perron identity, symmetry)."""
+    N, b, beta = 1 << 20, 64, 2.0
+    X = workloads.torus6(N, seed=42)
+    V = workloads.block(N, b, seed=1)
+    rows = workloads.row_sample(N, 96, seed=3)
+    rng = np.random.default_rng(5)
+    l = rng.uniform(0.5, 1.5, N).astype(np.float32) * 1e-3
+    r = rng.uniform(0.5, 1.5, N).astype(np.float32) * 1e-3
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
+    q, d, s, so, so2 = ctx.degree(beta, 1.0)
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    qo, sq = blocked.rows_apply_general(X, beta, None, rows=rows, want_rowsq=True)
+    assert np.abs(q.cpu().numpy()[rows] / qo[:, 0] - 1).max() <= TOL_DEG
+    t = lambda a: torch.from_numpy(a).to(dev)
+    Vd = fd.to_colmajor(V, dev)
+    Y = ctx.apply_general(beta, Vd, left=t(l), right=t(r))
+    ctx.synchronize()
+    Yo = blocked.rows_apply_general(X, beta, V, rows=rows, left=l, right=r)
+    assert relF(Y.cpu().numpy()[rows], Yo) <= TOL_APPLY
+    # M sqrt(d) = sqrt(d)
+    sd = torch.sqrt(d.double()).float()
+    W = torch.empty((b, N), dtype=torch.float32, device=dev).t()
+    W[:, 0] = sd
+    W[:, 1:] = Vd[:, 1:]
+    MW = ctx.apply(W)
+    ctx.synchronize()
+    assert float((MW[:, 0] - sd).abs().max() / sd.abs().max()) <= 2e-5
+    # U^T (M V) = (M U)^T V on two column pairs
+    MV = ctx.apply(Vd)
+    ctx.synchronize()
+    a = float((Vd[:, 2].double() * MV[:, 3].double()).sum())
+    bb = float((MV[:, 2].double() * Vd[:, 3].double()).sum())
+    scale = float(MV[:, 2].double().norm() * Vd[:, 3].double().norm())
+    assert abs(a - bb) <= 1e-5 * scale
+    ctx.close()
