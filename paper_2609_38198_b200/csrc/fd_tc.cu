@@ -46,6 +46,7 @@ struct TcParams {
     int64_t Nrow, N;             // valid rows / columns
     int num_work;                // row-pair tiles (256 rows each)
     int num_jt;                  // column tiles
+    int jt_chunk, num_chunks;    // the column range is swept in chunks small enough for L2 (block mode); all CTAs work on one chunk at a time
     int64_t np_rows;             // padded row count of the operand arrays (row index of K slab c = c * np + p)
     int64_t np_cols;
     int K16;
@@ -220,10 +221,14 @@ constexpr int kMaxBuf = 4;
 struct Barriers {
     uint64_t full[kStages], empty[kStages];
     uint64_t xfull, xempty;
-    uint64_t s_full[kMaxBuf];               // S tile ready in ring buffer (MMA -> warpgroup)
-    uint64_t s_done[kMaxBuf];               // block mode: P written in place; row-sum mode: S consumed (warpgroup -> MMA)
-    uint64_t p_half[kMaxBuf];               // block mode: first 64 columns of P written (lets the product MMA start early)
-    uint64_t kw_done[kMaxBuf];              // block mode: product MMAs that read P from this buffer have completed
+    // Ring-buffer barriers are indexed [buffer][row tile]: each one then has a single producer role and a single
+    // consumer role that waits on EVERY one of its phases.  (A parity wait is only unambiguous if the waiter has seen
+    // the previous phase complete; a barrier per buffer alone, shared by both row tiles, lets a waiter that skips
+    // alternate phases pass one phase early.)
+    uint64_t s_full[kMaxBuf][2];            // S tile ready in ring buffer (Gram issuer -> warpgroup)
+    uint64_t s_done[kMaxBuf][2];            // block mode: P written in place; row-sum mode: S consumed (warpgroup -> issuer)
+    uint64_t p_half[kMaxBuf][2];            // block mode: first 64 columns of P written (lets the product MMA start early)
+    uint64_t kw_done[kMaxBuf][2];           // block mode: product MMAs that read P from this buffer have completed
     uint64_t y_full[2], y_empty[2];         // accumulator flush hand-off (per row tile)
     uint32_t tmem_base;
     int abort_flag;
@@ -240,6 +245,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     extern __shared__ uint8_t smem_raw[];
     using SM = Smem<BT, MODE>;
     constexpr int NBUF = (MODE == kModeRowsum) ? 4 : 3;
+    constexpr uint32_t kRingPeriod = (NBUF & 1) ? 2 * NBUF : NBUF;   // tiles between two uses of a buffer by the same row tile
     constexpr uint32_t kYCol = 384;                    // block mode: Y_t at columns 384 + 64 t
     const int K16 = p.K16;
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -254,7 +260,11 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         // a column stage is released by the Gram issuer alone (row-sum mode) or by both product issuers (block mode)
         for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], MODE == kModeRowsum ? 1 : 2); }
         mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
-        for (int u = 0; u < kMaxBuf; ++u) { mbar_init(&bars->s_full[u], 1); mbar_init(&bars->s_done[u], 4); mbar_init(&bars->kw_done[u], 1); mbar_init(&bars->p_half[u], 4); }
+        for (int u = 0; u < kMaxBuf; ++u)
+            for (int t = 0; t < 2; ++t) {
+                mbar_init(&bars->s_full[u][t], 1); mbar_init(&bars->s_done[u][t], 4);
+                mbar_init(&bars->kw_done[u][t], 1); mbar_init(&bars->p_half[u][t], 4);
+            }
         for (int t = 0; t < 2; ++t) { mbar_init(&bars->y_full[t], 1); mbar_init(&bars->y_empty[t], 4); }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -268,9 +278,18 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
-    const int num_jt = p.num_jt;
-    const int tiles_per_item = 2 * num_jt;
-    const int my_items = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    // Work items of this CTA: (column chunk c, row-pair tile r) with c outermost, r = blockIdx.x + k * gridDim.x.  Every CTA
+    // sweeps chunk c for all of its rows before chunk c + 1, so the whole grid reads the same L2-sized slice of the
+    // column operands at about the same time; a row's partial results always come from the same threads, in order.
+    const int my_rows = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_items = my_rows * p.num_chunks;
+#define FD_ITEM_GEOMETRY(w)                                                                         \
+    const int cch = (w) / my_rows;                                                                  \
+    const int item = (int)blockIdx.x + ((w) % my_rows) * (int)gridDim.x;                            \
+    const int j0 = cch * p.jt_chunk;                                                                \
+    const int num_jt = (p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk;                   \
+    const int tiles_per_item = 2 * num_jt;                                                          \
+    (void)item; (void)tiles_per_item; (void)cch
     const int flush = p.flush;
 
     if (warp >= 8) {
@@ -283,7 +302,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             uint32_t it = 0;
             bool ok = true;
             for (int w = 0; w < my_items && ok; ++w) {
-                const int item = blockIdx.x + w * gridDim.x;
+                FD_ITEM_GEOMETRY(w);
                 ok = mbar_wait(&bars->xempty, (w & 1) ^ 1, abort_flag, p.status, 1);
                 if (!ok) break;
                 mbar_expect_tx(&bars->xfull, 2 * K16 * SM::kXChunk);
@@ -298,14 +317,14 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     uint8_t* st = stage_base + s * SM::stage_bytes(K16);
                     mbar_expect_tx(&bars->full[s], SM::stage_bytes(K16));
                     for (int c = 0; c < K16; ++c)
-                        tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)j * 128), &bars->full[s]);
+                        tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)(j0 + j) * 128), &bars->full[s]);
                     if (MODE != kModeRowsum) {
                         uint8_t* wst = st + K16 * SM::kXChunk;
-                        tma_load_2d(wst, &map_whi, j * 128, 0, &bars->full[s]);
-                        tma_load_2d(wst + SM::kWHalf, &map_whi, j * 128 + 64, 0, &bars->full[s]);
+                        tma_load_2d(wst, &map_whi, (j0 + j) * 128, 0, &bars->full[s]);
+                        tma_load_2d(wst + SM::kWHalf, &map_whi, (j0 + j) * 128 + 64, 0, &bars->full[s]);
                         if (MODE == kModeBlock) {
-                            tma_load_2d(wst + 2 * SM::kWHalf, &map_wlo, j * 128, 0, &bars->full[s]);
-                            tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, j * 128 + 64, 0, &bars->full[s]);
+                            tma_load_2d(wst + 2 * SM::kWHalf, &map_wlo, (j0 + j) * 128, 0, &bars->full[s]);
+                            tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, (j0 + j) * 128 + 64, 0, &bars->full[s]);
                         }
                     }
                 }
@@ -326,8 +345,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             constexpr uint32_t idesc_g = idesc_f16(128);
             uint32_t it0 = 0, gn0 = 0;
             bool ok = true;
-            uint64_t* free_bar = (MODE == kModeRowsum) ? bars->s_done : bars->kw_done;
             for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_GEOMETRY(w);
                 ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
                 if (!ok) break;
                 tc_fence_after();
@@ -337,8 +356,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const uint32_t itj = it0 + (uint32_t)(n >> 1);
                     const int s = itj % kStages;
                     if (w == 0) FD_TRACE(3, n, 0);
-                    ok = mbar_wait(&free_bar[buf], ((g / NBUF) & 1) ^ 1, abort_flag, p.status, 5);
-                    if (!ok) break;
+                    if (g >= (uint32_t)NBUF) {
+                        // the tile that used this buffer last (NBUF tiles ago, possibly of the other row tile) must be finished
+                        const uint32_t gp = g - NBUF;
+                        uint64_t* fb = (MODE == kModeRowsum) ? &bars->s_done[buf][gp & 1] : &bars->kw_done[buf][gp & 1];
+                        ok = mbar_wait(fb, (gp / kRingPeriod) & 1, abort_flag, p.status, 5);
+                        if (!ok) break;
+                    }
                     if (w == 0) FD_TRACE(3, n, 1);
                     if ((n & 1) == 0) {
                         ok = mbar_wait(&bars->full[s], (itj / kStages) & 1, abort_flag, p.status, 4);
@@ -361,7 +385,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
                         mma_ss(s_addr, a, b, idesc_g, 1);
                     }
-                    tc_commit(&bars->s_full[buf]);
+                    tc_commit(&bars->s_full[buf][n & 1]);
                     if (w == 0) FD_TRACE(3, n, 2);
                     if (MODE == kModeRowsum && (n & 1)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
                 }
@@ -380,12 +404,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             bool ok = true;
             const uint32_t y_addr = tmem + kYCol + 64 * t;
             for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_GEOMETRY(w);
                 for (int j = 0; j < num_jt && ok; ++j) {
                     const uint32_t g = gn0 + 2u * (uint32_t)j + (uint32_t)t;
                     const int buf = g % NBUF;
                     const int s = (it0 + (uint32_t)j) % kStages;
                     if (w == 0) FD_TRACE(0, 2 * j + t, 0);
-                    ok = mbar_wait(&bars->p_half[buf], (g / NBUF) & 1, abort_flag, p.status, 7);
+                    ok = mbar_wait(&bars->p_half[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 7);
                     if (!ok) break;
                     const bool group_start = (j % flush) == 0;
                     const bool group_end = ((j + 1) % flush) == 0 || j + 1 == num_jt;
@@ -405,7 +430,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         if (ks == 4) {
-                            ok = mbar_wait(&bars->s_done[buf], (g / NBUF) & 1, abort_flag, p.status, 7);
+                            ok = mbar_wait(&bars->s_done[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 7);
                             if (!ok) break;
                             tc_fence_after();
                         }
@@ -419,7 +444,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     }
                     if (!ok) break;
                     if (w == 0) FD_TRACE(0, 2 * j + t, 2);
-                    tc_commit(&bars->kw_done[buf]);
+                    tc_commit(&bars->kw_done[buf][t]);
                     if (group_end) { tc_commit(&bars->y_full[t]); ++n_grp; }
                     tc_commit(&bars->empty[s]);
                     if (w == 0) FD_TRACE(0, 2 * j + t, 3);
@@ -440,14 +465,14 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         bool ok = true;
 
         for (int w = 0; w < my_items && ok; ++w) {
-            const int item = blockIdx.x + w * gridDim.x;
+            FD_ITEM_GEOMETRY(w);
             const int64_t row = (int64_t)item * 256 + t * 128 + row_in_tile;
             if (MODE == kModeRowsum) {
                 double dsum = 0.0, dsq = 0.0;
                 for (int j = 0; j < num_jt && ok; ++j) {
                     const uint32_t g = gn0 + 2u * j + t;
                     const int buf = g % NBUF;
-                    ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 8);
+                    ok = mbar_wait(&bars->s_full[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 8);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t addr = tmem + lane_addr + 128u * buf;
@@ -459,7 +484,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     // the buffer can be refilled as soon as its values are in registers
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->s_done[buf]);
+                    if (lane == 0) mbar_arrive(&bars->s_done[buf][t]);
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
 #pragma unroll
@@ -513,7 +538,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const uint32_t g = gn0 + 2u * j + t;
                     const int buf = g % NBUF;
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 0);
-                    ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 9);
+                    ok = mbar_wait(&bars->s_full[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 9);
                     if (!ok) break;
                     tc_fence_after();
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 1);
@@ -549,14 +574,14 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                             tmem_wait_st();
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(&bars->p_half[buf]);
+                            if (lane == 0) mbar_arrive(&bars->p_half[buf][t]);
                         }
                     }
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 3);
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->s_done[buf]);
+                    if (lane == 0) mbar_arrive(&bars->s_done[buf][t]);
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 4);
                     // flush of the accumulator group that ended with the PREVIOUS tile of this row tile (its product
                     // MMA has had a whole tile of time to finish); the last group of the work item is flushed at once
@@ -571,7 +596,11 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const float l = p.left ? p.left[row] : 1.0f;
 #pragma unroll
                     for (int c = 0; c < BT; ++c)
-                        if (c < p.b) p.Y[row + (int64_t)c * p.ldy] = acc[c] * l * p.colscale_inv[c];
+                        if (c < p.b) {
+                            float* o = p.Y + row + (int64_t)c * p.ldy;
+                            const float v = acc[c] * l * p.colscale_inv[c];
+                            *o = cch == 0 ? v : *o + v;          // later column chunks add to the partial result of the same thread
+                        }
                 }
             }
             gn0 += (uint32_t)tiles_per_item;
@@ -787,6 +816,10 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.Nrow = a.Nrow; p.N = N;
     p.num_work = (int)ceil_div(a.Nrow, 256);
     p.num_jt = (int)ceil_div(N, 128);
+    // column chunk: ~1024 tiles (40 MB of fp16 operands at b = 64) stay resident in the 126 MB L2 while every CTA sweeps them
+    p.jt_chunk = rowsum ? p.num_jt : (c->opt_jt_chunk > 0 ? c->opt_jt_chunk : 1024);
+    if (p.jt_chunk > p.num_jt) p.jt_chunk = p.num_jt;
+    p.num_chunks = (int)ceil_div(p.num_jt, p.jt_chunk);
     p.np_rows = NP; p.np_cols = NP; p.K16 = K16;
     p.left = a.left; p.status = status;
     p.dbg = c->opt_trace >> 1;
