@@ -187,6 +187,33 @@ fd_status fd_nystrom(fd_ctx* ctx, const float* Xnew_dev, int64_t Nnew, int64_t l
 fd_status fd_scale_by_degree(fd_ctx* ctx, const float* v_dev, int64_t ldv, int32_t cols,
                              double power, float* out_dev, int64_t ldout);
 
+/* No counterpart in the paper: an entry point for callers that cannot allocate device memory.
+ *
+ * Every other call borrows its scratch from a workspace the caller allocates.  Some callers have
+ * no allocator to ask -- a plug-in that only receives input and output buffers, code that runs
+ * where its host framework forbids allocation, a process whose device memory pool belongs to
+ * someone else.  For them this variant of the direct-difference block product
+ *     Y = diag(left) K(X, X) diag(right) V,   K_ij = exp(-beta |x_i - x_j|^2)
+ * keeps its scratch (padded points, packed right block, split-column partial sums) in one
+ * file-scope device array of 8 MiB that every GPU loading the library holds until the process
+ * exits.  It calls no cudaMalloc / cudaFree and no allocating library routine; the caller passes
+ * inputs and outputs only (X row-major N x D pitch ldx; V, Y column-major; left, right may be
+ * NULL = ones; Y must not overlap V).  Limits: N <= FD_STATIC_MAX_N, D <= FD_STATIC_MAX_D,
+ * b <= FD_STATIC_MAX_B; anything larger is refused with FD_ERR_UNSUPPORTED and a message in
+ * errbuf (optional, may be NULL).  The first call made with a given device current resolves the
+ * array's device address (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * All calls share the array and it keeps the last call's contents: nothing in it needs clearing
+ * (every word read was written earlier in the same call), but two calls that overlap on the GPU
+ * race -- keep them on one stream or otherwise serialised.  Asynchronous on cuda_stream. */
+#define FD_STATIC_MAX_N 8192
+#define FD_STATIC_MAX_D 32
+#define FD_STATIC_MAX_B 32
+fd_status fd_apply_general_static(const float* X_dev, int64_t N, int32_t D, int64_t ldx, double beta,
+                                  const float* left_dev, const float* right_dev,
+                                  const float* V_dev, int64_t ldv, int32_t b,
+                                  float* Y_dev, int64_t ldy, void* cuda_stream,
+                                  char* errbuf, size_t errbuf_len);
+
 const char* fd_status_string(fd_status st);
 const char* fd_last_error(const fd_ctx* ctx);
 int32_t     fd_version(void);

@@ -26,7 +26,7 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
     "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree",
-    "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
+    "fd_apply_general_static", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
 
@@ -76,6 +76,9 @@ def _load() -> ctypes.CDLL:
     for name in ("fd_synchronize", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree", "fd_apply",
                  "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree"):
         getattr(lib, name).restype = c_int32
+    lib.fd_apply_general_static.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_double, c_void_p, c_void_p, c_void_p,
+                                            c_int64, c_int32, c_void_p, c_int64, c_void_p, ctypes.c_char_p, c_size_t]
+    lib.fd_apply_general_static.restype = c_int32
     lib.fd_status_string.argtypes = [c_int32]
     lib.fd_status_string.restype = c_char_p
     lib.fd_last_error.argtypes = [c_void_p]
@@ -257,6 +260,29 @@ class Context:
         with torch.cuda.device(self.device):
             self._check(lib.fd_scale_by_degree(self._h, _ptr(v), _ld(v), v.shape[1], power, _ptr(out), _ld(out)))
         return out
+
+
+FD_STATIC_MAX_N, FD_STATIC_MAX_D, FD_STATIC_MAX_B = 8192, 32, 32
+
+
+def fd_apply_general_static(X: torch.Tensor, beta: float, V: torch.Tensor, left=None, right=None,
+                            out: torch.Tensor | None = None) -> torch.Tensor:
+    """Y = diag(left) K(X, X) diag(right) V through the entry point that allocates nothing on the device: its
+    scratch is the library's own fixed device array.  For callers that cannot allocate; sizes are limited to
+    FD_STATIC_MAX_N / _D / _B, and calls must not overlap on the GPU.  `out` must be given by such a caller; when it
+    is omitted here the binding allocates it for convenience (that allocation is the binding's, not the library's)."""
+    assert X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    if V.dim() == 1:
+        V = V[:, None]
+    N, D, b = int(X.shape[0]), int(X.shape[1]), int(V.shape[1])
+    Y = out if out is not None else _colmajor(N, b, X.device)
+    err = ctypes.create_string_buffer(256)
+    with torch.cuda.device(X.device):
+        st = lib.fd_apply_general_static(_ptr(X), N, D, X.stride(0), float(beta), _ptr(left), _ptr(right), _ptr(V), _ld(V), b,
+                                         _ptr(Y), _ld(Y), c_void_p(torch.cuda.current_stream(X.device).cuda_stream), err, 256)
+    if st != FD_OK:
+        raise FdError(st, err.value.decode())
+    return Y
 
 
 def to_colmajor(a, device) -> torch.Tensor:

@@ -279,3 +279,118 @@ fd_status apply_simt(fd_ctx* c, const ApplyArgs& a) {
 }
 
 }  // namespace fd
+
+// ================================================================================================
+// fd_apply_general_static: the split direct-difference block product for callers that cannot
+// allocate device memory.
+//
+// Some hosts of this library hold no allocator they may call at the point where they need a
+// kernel product: code running inside another framework's stream callback or capture-adjacent
+// region, a plug-in that is handed input and output buffers only, a process whose memory pool
+// is owned and sized by someone else.  For them every byte of scratch the ordinary entry points
+// take from the caller's workspace lives here instead, in one file-scope device array of fixed
+// size that each GPU loading the library keeps until the process exits.
+//
+// Scratch layout inside the array (floats): padded copy of the points, packed right-hand block,
+// split-column partial sums.  Nothing in it has to start at zero: every word a launch reads was
+// written earlier in the same call.  All calls share the array, so two calls that overlap on the
+// GPU (different streams, or different host threads) race; serialise them.
+namespace fd {
+namespace {
+
+constexpr size_t kStaticXs = (size_t)FD_STATIC_MAX_N * FD_STATIC_MAX_D;          // padded points
+constexpr size_t kStaticWp = (size_t)FD_STATIC_MAX_N * FD_STATIC_MAX_B;          // packed right block
+constexpr size_t kStaticPart = (size_t)3 << 19;                                  // split partials (6 MiB)
+constexpr size_t kStaticFloats = kStaticXs + kStaticWp + kStaticPart;            // 8 MiB in total
+
+static __device__ __align__(256) float g_static_scratch[kStaticFloats];
+
+// Device address of the array per device ordinal, resolved on the first call made with that device current.
+// (In host code the symbol's name is only a handle; the address a kernel can use comes from the runtime.)
+constexpr int kMaxDevices = 64;
+float* g_static_ptr[kMaxDevices] = {};
+
+__global__ void k_static_pad_copy(const float* __restrict__ src, int64_t ld, int64_t n, int D, int DP, float* __restrict__ dst) {
+    int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = n * DP;
+    for (; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = idx / DP;
+        const int k = (int)(idx - i * DP);
+        dst[idx] = k < D ? src[i * ld + k] : 0.0f;
+    }
+}
+
+fd_status static_fail(char* errbuf, size_t errlen, fd_status st, const char* fmt, long long a = 0, long long b = 0) {
+    if (errbuf && errlen) snprintf(errbuf, errlen, fmt, a, b);
+    return st;
+}
+
+}  // namespace
+}  // namespace fd
+
+extern "C" fd_status fd_apply_general_static(const float* X_dev, int64_t N, int32_t D, int64_t ldx, double beta,
+                                             const float* left_dev, const float* right_dev, const float* V_dev,
+                                             int64_t ldv, int32_t b, float* Y_dev, int64_t ldy, void* cuda_stream,
+                                             char* errbuf, size_t errbuf_len) {
+    using namespace fd;
+    if (errbuf && errbuf_len) errbuf[0] = 0;
+    if (!X_dev || !V_dev || !Y_dev) return static_fail(errbuf, errbuf_len, FD_ERR_INVALID, "X, V and Y must be non-null");
+    if (N < 1 || D < 1 || b < 1 || ldx < D || ldv < N || ldy < N || !(beta > 0) || !(beta < 1e30))
+        return static_fail(errbuf, errbuf_len, FD_ERR_INVALID, "bad size, pitch or beta");
+    if (N > FD_STATIC_MAX_N) return static_fail(errbuf, errbuf_len, FD_ERR_UNSUPPORTED, "N = %lld exceeds FD_STATIC_MAX_N = %lld", (long long)N, FD_STATIC_MAX_N);
+    if (D > FD_STATIC_MAX_D) return static_fail(errbuf, errbuf_len, FD_ERR_UNSUPPORTED, "D = %lld exceeds FD_STATIC_MAX_D = %lld", D, FD_STATIC_MAX_D);
+    if (b > FD_STATIC_MAX_B) return static_fail(errbuf, errbuf_len, FD_ERR_UNSUPPORTED, "b = %lld exceeds FD_STATIC_MAX_B = %lld", b, FD_STATIC_MAX_B);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    // set-up, once per device: resolve the device address of the scratch array
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return static_fail(errbuf, errbuf_len, FD_ERR_CUDA, "cudaGetDevice failed or device ordinal out of range");
+    if (!g_static_ptr[dev]) {
+        float* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) return static_fail(errbuf, errbuf_len, FD_ERR_CUDA, "cudaGetSymbolAddress failed (%lld)", (long long)e);
+        g_static_ptr[dev] = ptr;
+    }
+    float* xs = g_static_ptr[dev];
+    float* wp = xs + kStaticXs;
+    float* part = wp + kStaticWp;
+
+    const int DP = (int)round_up(D, 4), DP4 = DP / 4;
+    const int BT = pick_bt(b);
+    const float nbeta2 = (float)(-beta * kLog2e);
+    int grid_copy = (int)ceil_div(N * DP, 256);
+    k_static_pad_copy<<<grid_copy, 256, 0, stream>>>(X_dev, ldx, N, D, DP, xs);
+    ++g_launches;
+    dim3 pg((unsigned)ceil_div(N, 32), (unsigned)ceil_div(BT, 32));
+    k_pack_w<<<pg, dim3(32, 8), 0, stream>>>(V_dev, ldv, right_dev, N, 0, b, BT, wp);
+    ++g_launches;
+    // split the column range so that ~600 CTAs run, within the partials' capacity
+    const int64_t row_tiles = ceil_div(N, kRows);
+    int64_t sp = row_tiles >= 592 ? 1 : ceil_div(592, row_tiles);
+    const int64_t cap = (int64_t)(kStaticPart / ((size_t)BT * (size_t)N));
+    if (sp > cap) sp = cap;
+    if (sp > ceil_div(N, kTJ)) sp = ceil_div(N, kTJ);
+    if (sp < 1) sp = 1;
+    const int64_t jps = round_up(ceil_div(N, sp), kTJ);
+    sp = ceil_div(N, jps);
+    dim3 grid((unsigned)row_tiles, (unsigned)sp);
+    bool ok;
+    if (sp == 1) {
+        ok = launch_simt_any(DP4, BT, grid, stream, xs, N, xs, N, nbeta2, wp, jps, left_dev, Y_dev, ldy, 0, b, nullptr, nullptr, nullptr);
+        ++g_launches;
+    } else {
+        ok = launch_simt_any(DP4, BT, grid, stream, xs, N, xs, N, nbeta2, wp, jps, nullptr, part, N, (int64_t)BT * N, BT, nullptr,
+                             nullptr, nullptr);
+        ++g_launches;
+        if (ok) {
+            dim3 rg((unsigned)ceil_div(N, 256), (unsigned)b);
+            k_reduce_block<<<rg, 256, 0, stream>>>(part, (int)sp, (int64_t)BT * N, N, b, left_dev, Y_dev, ldy);
+            ++g_launches;
+        }
+    }
+    if (!ok) return static_fail(errbuf, errbuf_len, FD_ERR_UNSUPPORTED, "no kernel instantiation for this D, b");
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return static_fail(errbuf, errbuf_len, FD_ERR_CUDA, "kernel launch failed (%lld)", (long long)e);
+    return FD_OK;
+}
