@@ -37,7 +37,7 @@ MUFU_PER_CLK_SM = 16
 FMA_PER_CLK_SM = 128
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None.
-NCU_TRAFFIC_BYTES = {"simt": None, "tc": None}
+NCU_TRAFFIC_BYTES = {"simt": None, "tc": 45.9e9 + 2.19e9}   # k_tc block mode at N = 2^20, profiles/bench_c5_n2e20_launch_list.md
 
 
 def measured_peaks():
@@ -278,7 +278,8 @@ def run_gpu(args):
         roofline = {"bound": "alu", "kernel": "block product Y = M V (dominant kernel)", "binder": binder,
                     "achieved": pairs_per_s / 1e9, "peak": peak_pairs / 1e9, "unit": "Gpairs/s",
                     "frac": pairs_per_s / peak_pairs, "peak_source": f"unit counts x {peak_kind} max SM clock",
-                    "mufu_floor_frac": pairs_per_s / mufu_peak, "traffic": NCU_TRAFFIC_BYTES.get(path_used),
+                    "mufu_floor_frac": pairs_per_s / mufu_peak, "traffic": NCU_TRAFFIC_BYTES.get(path_used) if N == (1 << 20) else None,
+                    "algorithmic_bytes": 4.0 * N * (D + 2 * b + 2),
                     "sm_mhz_seen": mhz}
         out = {"metric": METRIC, "value": units * world / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
