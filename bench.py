@@ -158,6 +158,21 @@ def run_reference(args):
     print(json.dumps(out), flush=True)
 
 
+# ------------------------------------------------------------------------------------------- multi-rank plumbing
+def max_over_ranks(values, dist, device):
+    """Device-side times of every rank -> their maximum over ranks (the job is as slow as its slowest replica)."""
+    import torch
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_value(units_per_rank: float, world: int, ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling): all units over the slowest rank's time."""
+    return units_per_rank * world / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------- GPU arm
 def run_gpu(args):
     import torch
@@ -253,10 +268,7 @@ def run_gpu(args):
     barrier()
     e2e_ms = e_a.elapsed_time(e_b) / e2e_steps
 
-    t = torch.tensor([total_ms, e2e_ms, deg_ms, app_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms, deg_ms, app_ms = [float(v) for v in t.cpu()]
+    total_ms, e2e_ms, deg_ms, app_ms = max_over_ranks([total_ms, e2e_ms, deg_ms, app_ms], dist, dev)
     step_ms = total_ms / args.steps
     units = float(N) * N * (b + 2)
 
@@ -281,21 +293,64 @@ def run_gpu(args):
                     "mufu_floor_frac": pairs_per_s / mufu_peak, "traffic": NCU_TRAFFIC_BYTES.get(path_used) if N == (1 << 20) else None,
                     "algorithmic_bytes": 4.0 * N * (D + 2 * b + 2),
                     "sm_mhz_seen": mhz}
-        out = {"metric": METRIC, "value": units * world / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        out = {"metric": METRIC, "value": job_value(units, world, step_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
                "apply_only": {"ms": app_ms, "pair_cols_per_s": float(N) * N * b / (app_ms * 1e-3), "pairs_per_s": pairs_per_s},
                "degree_ms": deg_ms, "path": path_used, "roofline": roofline,
-               "e2e": {"value": units * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "e2e": {"value": job_value(units, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(Xh.numel() * 4 + Vh.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 4)},
                "gpu_launches": int(launches), "workspace_bytes": ctx.workspace_bytes}
-        if not args.no_cpu and world == 1 or (not args.no_cpu and rank == 0):
+        if not args.no_cpu:
             out["cpu_baseline"] = cpu_baseline(X, V, cfg)
+        ctx.close()
+        if not args.no_eigs:
+            del Xd, Vd, Yd
+            torch.cuda.empty_cache()
+            out["time_to_k_eigs"] = time_to_k_eigs(fd, dev, full=args.eigs_full)
         print(json.dumps(out), flush=True)
     ctx.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def time_to_k_eigs(fd, dev, full=False):
+    """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs), and the whole
+    dyadic bandwidth flow, on the 6-torus workloads (C3: N = 2^17, b = 32, k = 64; with --eigs-full also C5: N = 2^20,
+    b = 64, k = 128).  Host wall clock around synchronous calls."""
+    import torch
+    import workloads
+    res = []
+    cases = [("C3", 1 << 17, 64, 32)] + ([("C5", 1 << 20, 128, 64)] if full else [])
+    for name, N, k, b in cases:
+        X = torch.from_numpy(workloads.torus6(N, seed=42)).to(dev)
+        m_max = (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
+        ctx = fd.Context(X, b_max=b, m_max=m_max)
+        ctx.degree(2.0, 1.0)                                         # warm-up of both passes
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        ctx.degree(2.0, 1.0)
+        t1 = time.perf_counter()
+        lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=400, allow_not_converged=True)
+        t2 = time.perf_counter()
+        rec = {"workload": f"{name}: 6-torus N={N}, k={k}, b={b}, alpha=1, beta=2.0, tol=1e-6", "degree_s": t1 - t0,
+               "eigs_s": t2 - t1, "total_s": t2 - t0, "applies": int(info.applies), "restarts": int(info.restarts),
+               "converged": int(info.converged), "of": k + 1, "max_residual": float(info.max_residual),
+               "seconds_in_apply": float(info.seconds_apply), "lambda_1": float(lam[1]), "lambda_k": float(lam[k])}
+        if name == "C3":
+            t3 = time.perf_counter()
+            bx, outcome, lam2, U2, recs = ctx.beta_flow(k, b, 1.0, beta_start=1.0, beta_max=1000.0, tol=1e-6, max_applies=400)
+            t4 = time.perf_counter()
+            rec["flow"] = {"grid": "beta = 1, 2, 4, ... <= 1000 (dyadic), warm-started probes", "seconds": t4 - t3,
+                           "beta_x": bx, "outcome": outcome, "probes": len(recs),
+                           "applies": int(sum(r["applies"] for r in recs)), "n_eff_at_beta_x": recs[-1]["n_eff"],
+                           "d_hat_at_beta_x": recs[-1]["d_hat"]}
+        ctx.close()
+        del ctx, X
+        torch.cuda.empty_cache()
+        res.append(rec)
+    return res
 
 
 def cpu_baseline(X, V, cfg):
@@ -325,6 +380,8 @@ def main():
     ap.add_argument("--n", type=int, default=20, help="log2 of the number of points (default 20: the headline size)")
     ap.add_argument("--path", default="", choices=["", "auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
+    ap.add_argument("--no-eigs", action="store_true", help="skip the time-to-k-eigenpairs leg")
+    ap.add_argument("--eigs-full", action="store_true", help="also time the eigensolve at N = 2^20 (k = 128, b = 64)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = max(args.warmup, 3)

@@ -148,7 +148,8 @@ typedef struct {
     double beta, S_off, S_off_2beta, n_eff, d_hat, V_bias, V_stat, V_mach, V, g_P;
     double lambda1;            /* first nontrivial eigenvalue                                 */
     int32_t applies;           /* block applies the probe's eigensolve took                   */
-    int32_t flags;             /* bit 0: inadmissible (Eq. 12); bit 1: final (vertex) probe   */
+    int32_t flags;             /* bit 0: inadmissible (Eq. 12); bit 1: final (vertex) probe;  */
+                               /* bit 2: eigensolve stalled above tol (residuals <= 1e-4)     */
 } fd_probe;
 
 typedef struct {

@@ -229,6 +229,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
     int nsel = 0, nconv = 0;
     fd_status final_status = FD_ERR_NOT_CONVERGED;
     int stagnation = 0;
+    // stagnation of the residuals at the accuracy floor of the fp32 operator (noise-smeared spectra): stop early
+    double best_res = 1e300;
+    int since_best = 0;
 
     for (int iter = 0;; ++iter) {
         const int m = S.m;
@@ -284,6 +287,15 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         for (int i = 0; i < std::min(nwant, nsel); ++i) all = all && resid[i] <= thr;
         if (all) { final_status = FD_OK; break; }
         if (S.applies >= max_applies) break;
+        {
+            double worst = 0.0;
+            for (int i = 0; i < std::min(nwant, nsel); ++i) worst = std::max(worst, resid[i]);
+            if (nsel >= nwant && worst < 0.9 * best_res) { best_res = worst; since_best = 0; }
+            else if (nsel >= nwant) ++since_best;
+            // the largest wanted residual has not improved by 10 % over 12 expansions and is within 30x of the target:
+            // the operator's own rounding error is the floor; more applies do not help
+            if (since_best >= 12 && best_res <= 30.0 * thr) break;
+        }
         if (m >= N) break;                                        // basis spans everything: nothing more to add
 
         // ---- choose the expansion columns: largest residuals first ------------------------------
