@@ -83,7 +83,9 @@ fd_status fd_destroy(fd_ctx* ctx);
  * between accumulator flushes of the tensor-core kernel), "tc_max_mag" (largest beta * log2(e) *
  * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "poly_exp" (share
  * of exponentials sent to the FMA pipe, 0..1), "trace" (tuning aid: the tensor-core kernel stamps
- * clock values of its first tiles into scratch).  fd_get_option also reports "last_path" (the
+ * clock values of its first tiles into scratch), "wait_selftest" (value = limit in SM cycles: enqueues
+ * a one-thread kernel whose bounded wait on a barrier that nothing completes must expire; the next
+ * fd_synchronize then returns FD_ERR_TIMEOUT and the context stays usable).  fd_get_option also reports "last_path" (the
  * family that served the latest pass), "beta", "mean_sq", "max_sq".  Unknown name -> FD_ERR_INVALID. */
 fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
 fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);

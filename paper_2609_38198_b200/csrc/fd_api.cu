@@ -152,6 +152,9 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "tc_max_mag")) {
         if (!(v > 0)) return fail(c, FD_ERR_INVALID, "tc_max_mag must be positive");
         c->opt_tc_max_mag = v;
+    } else if (!strcmp(name, "wait_selftest")) {
+        if (!(v >= 1000) || v > 4e9) return fail(c, FD_ERR_INVALID, "wait_selftest: limit in cycles, 1e3..4e9");
+        return tc_wait_selftest(c, (long long)v);
     } else if (!strcmp(name, "trace")) {
         c->opt_trace = (int)v;
     } else if (!strcmp(name, "poly_exp")) {

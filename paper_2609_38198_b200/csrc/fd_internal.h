@@ -119,6 +119,8 @@ bool tc_supported(const fd_ctx* c, const ApplyArgs& a);
 fd_status apply_dispatch(fd_ctx* c, const ApplyArgs& a);
 // Reads and clears the tensor-core kernel's status word; FD_ERR_TIMEOUT if a bounded wait expired.  Synchronises.
 fd_status tc_check_status(fd_ctx* c);
+// Launches a one-thread kernel whose bounded wait must expire after limit_cycles (test of the time-out plumbing).
+fd_status tc_wait_selftest(fd_ctx* c, long long limit_cycles);
 
 // ---- small kernels (fd_elementwise.cu) ------------------------------------------------------
 fd_status ew_pow(fd_ctx* c, const float* in, double p, float* out, int64_t n);            // out = in^p

@@ -92,7 +92,8 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: returns false (and raises the abort flag) when the limit is hit or another role aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, int code) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, int code,
+                                          long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
@@ -100,7 +101,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         __nanosleep(40);            // back off: many warps polling shared memory slow the MMA issuer down
         if ((++spins & 63) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 atomicCAS(status, 0u, (unsigned)(0x100 | code));
                 return false;
@@ -613,6 +614,19 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     }
 }
 
+// Exercises the bounded-wait path without any fault: one thread waits on a barrier that nothing will ever complete,
+// with a short limit; the wait gives up, records its code in the status word and the kernel returns normally.
+__global__ void k_wait_selftest(unsigned int* status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(&bar, 0, &abort_flag, status, 0x7f, limit_cycles);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ operand packing
 // Augmented fp16 hi|lo operand rows.  role 0 (rows of the product): [c x, e, 1]; role 1 (columns): [c x, 1, e] with
 // c = sqrt(2 b'), e = -b' |x - mu|^2 (+ extra_j: bias and log2 of a positive right vector for role 1).
@@ -861,6 +875,12 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
 #undef FD_TC_CASE
         }
     }
+    return FD_OK;
+}
+
+fd_status tc_wait_selftest(fd_ctx* c, long long limit_cycles) {
+    k_wait_selftest<<<1, 32, 0, c->stream>>>(c->at<unsigned int>(c->L.status), limit_cycles);
+    FD_LAUNCH_CHECK(c, "k_wait_selftest");
     return FD_OK;
 }
 

@@ -222,3 +222,21 @@ def test_full_size_sampled_rows_and_identities(fd, dev):
     scale = float(MV[:, 2].double().norm() * Vd[:, 3].double().norm())
     assert abs(a - bb) <= 1e-5 * scale
     ctx.close()
+
+
+def test_bounded_wait_expires_cleanly_and_context_survives(fd, dev):
+    # a wait on a barrier that nothing completes, with a 1 ms limit: the kernel returns, the status word reports it
+    X = workloads.torus6(1024, seed=2)
+    V = workloads.block(1024, 16, seed=1)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=16)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    ctx.degree(1.0, 1.0)
+    ctx.set_option("wait_selftest", 2.0e6)
+    with pytest.raises(fd.FdError) as e:
+        ctx.synchronize()
+    assert e.value.status == fd.FD_ERR_TIMEOUT and "0x17f" in str(e.value)
+    ctx.synchronize()                                  # reported once, then cleared
+    Y = ctx.apply(fd.to_colmajor(V, dev))              # the context (and the GPU) are still fine
+    ctx.synchronize()
+    assert relF(Y.cpu().numpy(), dense.apply(X, 1.0, 1.0, V)) <= TOL_APPLY
+    ctx.close()
