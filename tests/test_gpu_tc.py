@@ -240,3 +240,68 @@ def test_bounded_wait_expires_cleanly_and_context_survives(fd, dev):
     ctx.synchronize()
     assert relF(Y.cpu().numpy(), dense.apply(X, 1.0, 1.0, V)) <= TOL_APPLY
     ctx.close()
+
+
+def test_c4_full_size_sampled_rows(fd, dev):
+    """C4 at full size (N = 262144, D = 30: three 16-wide K slabs): sampled rows of q and of the general product against
+    the oracle; Perron identity of the normalised operator."""
+    N, b, beta = 262144, 32, 2.0
+    X = workloads.latent_torus(N, seed=42)
+    V = workloads.block(N, b, seed=1)
+    rows = workloads.row_sample(N, 64, seed=4)
+    rng = np.random.default_rng(6)
+    l = rng.uniform(0.5, 1.5, N).astype(np.float32) * 1e-3
+    r = rng.uniform(0.5, 1.5, N).astype(np.float32) * 1e-3
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
+    q, d, s, so, so2 = ctx.degree(beta, 1.0)
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    qo = blocked.rows_apply_general(X, beta, None, rows=rows)
+    assert np.abs(q.cpu().numpy()[rows] / qo[:, 0] - 1).max() <= TOL_DEG
+    t = lambda a: torch.from_numpy(a).to(dev)
+    Vd = fd.to_colmajor(V, dev)
+    Y = ctx.apply_general(beta, Vd, left=t(l), right=t(r))
+    ctx.synchronize()
+    Yo = blocked.rows_apply_general(X, beta, V, rows=rows, left=l, right=r)
+    assert relF(Y.cpu().numpy()[rows], Yo) <= TOL_APPLY
+    sd = torch.sqrt(d.double()).float()
+    W = torch.empty((b, N), dtype=torch.float32, device=dev).t()
+    W[:, 0] = sd
+    W[:, 1:] = Vd[:, 1:]
+    MW = ctx.apply(W)
+    ctx.synchronize()
+    assert float((MW[:, 0] - sd).abs().max() / sd.abs().max()) <= 2e-5
+    ctx.close()
+
+
+def test_c3_full_size_eigs_certificate(fd, dev):
+    """C3 at full size (N = 131072, b = 32, k = 64, beta = 2): no dense oracle is affordable, so the gates are the
+    properties that hold at any size: lambda_0 = 1 (Perron), eigenvalues in (0, 1] and descending, orthonormal vectors,
+    small residuals measured with an independent product (the direct-difference kernels), Perron vector = sqrt(d)."""
+    N, b, k, beta = 131072, 32, 64, 2.0
+    X = workloads.torus6(N, seed=42)
+    m_max = 320
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=m_max)
+    q, d, s, so, so2 = ctx.degree(beta, 1.0)
+    lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=300)
+    assert info.converged == k + 1
+    assert abs(lam[0] - 1.0) <= 1e-6
+    assert np.all(np.diff(lam) <= 1e-9) and lam[-1] > 0
+    G = (U.double().t() @ U.double()).cpu().numpy()
+    assert np.abs(G - np.eye(k + 1)).max() <= 1e-5
+    sd = torch.sqrt(d.double())
+    sd = sd / sd.norm()
+    assert float((U[:, 0].double().abs() - sd).abs().max()) <= 1e-4 * float(sd.max())
+    # residuals with the other kernel family (degree + product on the direct-difference path)
+    ctx2 = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
+    ctx2.set_option("path", fd.FD_PATH_SIMT)
+    ctx2.degree(beta, 1.0)
+    lam_t = torch.from_numpy(lam).to(dev)
+    worst = 0.0
+    for c0 in range(0, k + 1, b):
+        blk = U[:, c0:c0 + b].t().contiguous().t()
+        MU = ctx2.apply(blk)
+        ctx2.synchronize()
+        R = MU.double() - blk.double() * lam_t[c0:c0 + b][None, :]
+        worst = max(worst, float(R.norm(dim=0).max()))
+    assert worst <= 5e-6, worst
+    ctx.close(); ctx2.close()
