@@ -7,43 +7,70 @@ namespace fd {
 
 namespace {
 
-constexpr int kTnTile = 32;       // output tile of the A^T B kernel is 32 x 32
-constexpr int kTnRows = 64;       // rows staged per step
+constexpr int kTnI = 64;          // output tile of the A^T B kernel: 64 (columns of A) x 32 (columns of B)
+constexpr int kTnJ = 32;
+constexpr int kTnRows = 64;       // rows staged per step; one step is summed in fp32, steps are added in fp64
 
-// part[chunk][i + j * m1] = sum over this chunk's rows of A[r, i] * B[r, j], fp64 accumulation.
-__global__ void __launch_bounds__(256)
+// part[chunk][i + j * m1] = sum over this chunk's rows of A[r, i] * B[r, j].
+// 128 threads, each a 4 x 4 register tile.  Products of 64 consecutive rows are accumulated in fp32 (entries of
+// orthonormal columns are ~N^-1/2, so a 64-term partial sum loses ~1e-10 absolute) and every such partial sum is
+// added to an fp64 accumulator, which keeps the long sum over N rows at fp64 accuracy at fp32 FMA speed.
+__global__ void __launch_bounds__(128)
 k_tn_partial(const float* __restrict__ A, int64_t lda, int m1, const float* __restrict__ B, int64_t ldb, int m2,
              int64_t N, int64_t rows_per_chunk, double* __restrict__ part) {
-    __shared__ float sa[kTnRows][kTnTile + 1];
-    __shared__ float sb[kTnRows][kTnTile + 1];
-    const int ti = blockIdx.x * kTnTile, tj = blockIdx.y * kTnTile;
+    constexpr int PA = kTnI + 4, PB = kTnJ + 4;                 // padded pitches (keep float4 alignment)
+    __shared__ __align__(16) float sa[kTnRows * PA];
+    __shared__ __align__(16) float sb[kTnRows * PB];
+    const int ti0 = blockIdx.x * kTnI, tj0 = blockIdx.y * kTnJ;
     const int64_t r_beg = (int64_t)blockIdx.z * rows_per_chunk;
     const int64_t r_end = r_beg + rows_per_chunk < N ? r_beg + rows_per_chunk : N;
-    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;      // thread computes (2 x 2) at (2 tx.., 2 ty..)
-    double acc00 = 0, acc01 = 0, acc10 = 0, acc11 = 0;
+    const int ti = threadIdx.x & 15, tj = threadIdx.x >> 4;     // i0 = 4 ti, j0 = 4 tj
+    double acc[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.0;
     for (int64_t r0 = r_beg; r0 < r_end; r0 += kTnRows) {
         __syncthreads();
-        for (int t = threadIdx.x; t < kTnRows * kTnTile; t += 256) {
-            int rr = t % kTnRows, cc = t / kTnRows;               // rows fastest: coalesced along a column
-            int64_t r = r0 + rr;
-            sa[rr][cc] = (r < r_end && ti + cc < m1) ? A[r + (int64_t)(ti + cc) * lda] : 0.f;
-            sb[rr][cc] = (r < r_end && tj + cc < m2) ? B[r + (int64_t)(tj + cc) * ldb] : 0.f;
+        for (int t = threadIdx.x; t < kTnRows * kTnI; t += 128) {
+            const int rr = t % kTnRows, cc = t / kTnRows;       // rows fastest: coalesced along a column
+            const int64_t r = r0 + rr;
+            sa[rr * PA + cc] = (r < r_end && ti0 + cc < m1) ? A[r + (int64_t)(ti0 + cc) * lda] : 0.f;
+        }
+        for (int t = threadIdx.x; t < kTnRows * kTnJ; t += 128) {
+            const int rr = t % kTnRows, cc = t / kTnRows;
+            const int64_t r = r0 + rr;
+            sb[rr * PB + cc] = (r < r_end && tj0 + cc < m2) ? B[r + (int64_t)(tj0 + cc) * ldb] : 0.f;
         }
         __syncthreads();
+        float f[4][4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) f[u][v] = 0.f;
 #pragma unroll 8
         for (int rr = 0; rr < kTnRows; ++rr) {
-            double a0 = sa[rr][2 * tx], a1 = sa[rr][2 * tx + 1];
-            double b0 = sb[rr][2 * ty], b1 = sb[rr][2 * ty + 1];
-            acc00 = fma(a0, b0, acc00); acc01 = fma(a0, b1, acc01);
-            acc10 = fma(a1, b0, acc10); acc11 = fma(a1, b1, acc11);
+            const float4 a = *reinterpret_cast<const float4*>(&sa[rr * PA + 4 * ti]);
+            const float4 b = *reinterpret_cast<const float4*>(&sb[rr * PB + 4 * tj]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) f[u][v] = fmaf(av[u], bv[v], f[u][v]);
         }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] += (double)f[u][v];
     }
     double* o = part + (size_t)blockIdx.z * m1 * m2;
-    int i0 = ti + 2 * tx, j0 = tj + 2 * ty;
-    if (i0 < m1 && j0 < m2) o[i0 + (size_t)j0 * m1] = acc00;
-    if (i0 < m1 && j0 + 1 < m2) o[i0 + (size_t)(j0 + 1) * m1] = acc01;
-    if (i0 + 1 < m1 && j0 < m2) o[i0 + 1 + (size_t)j0 * m1] = acc10;
-    if (i0 + 1 < m1 && j0 + 1 < m2) o[i0 + 1 + (size_t)(j0 + 1) * m1] = acc11;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int i = ti0 + 4 * ti + u, j = tj0 + 4 * tj + v;
+            if (i < m1 && j < m2) o[i + (size_t)j * m1] = acc[u][v];
+        }
 }
 
 __global__ void k_tn_reduce(const double* __restrict__ part, int chunks, int64_t mm, double* __restrict__ out) {
@@ -137,8 +164,8 @@ fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float
     if (chunks < 1) return fail(c, FD_ERR_WORKSPACE, "projection scratch too small for %d x %d", m1, m2);
     int64_t rpc = round_up(ceil_div(N, chunks), kTnRows);
     chunks = ceil_div(N, rpc);
-    dim3 grid((unsigned)ceil_div(m1, kTnTile), (unsigned)ceil_div(m2, kTnTile), (unsigned)chunks);
-    k_tn_partial<<<grid, 256, 0, c->stream>>>(A, lda, m1, B, ldb, m2, N, rpc, scratch);
+    dim3 grid((unsigned)ceil_div(m1, kTnI), (unsigned)ceil_div(m2, kTnJ), (unsigned)chunks);
+    k_tn_partial<<<grid, 128, 0, c->stream>>>(A, lda, m1, B, ldb, m2, N, rpc, scratch);
     FD_LAUNCH_CHECK(c, "k_tn_partial");
     k_tn_reduce<<<(unsigned)ceil_div((int64_t)mm, 256), 256, 0, c->stream>>>(scratch, (int)chunks, (int64_t)mm, out_dev);
     FD_LAUNCH_CHECK(c, "k_tn_reduce");

@@ -17,6 +17,8 @@
 #include <algorithm>
 #include <chrono>
 #include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <vector>
 
 #include "fd_dense.h"
@@ -233,8 +235,10 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
     double best_res = 1e300;
     int since_best = 0;
 
+    double t_rr = 0, t_eig = 0, t_res = 0, t_restart = 0, t_orth = 0, t_ext = 0;
     for (int iter = 0;; ++iter) {
         const int m = S.m;
+        auto tp0 = clk::now();
         // ---- Rayleigh-Ritz with first-order correction for G = Q^T Q = I + E ---------------------
         // Tc = T - (E T + T E) / 2 with E = G - I; T E = (E T)^T because both are symmetric
         std::vector<double> Tc((size_t)m * m), ET((size_t)m * m, 0.0);
@@ -250,7 +254,10 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             for (int i = 0; i < m; ++i)
                 Tc[i + (size_t)j * m] = S.T[i + (size_t)j * m_cap] - 0.5 * (ET[i + (size_t)j * m] + ET[j + (size_t)i * m]);
         std::vector<double> lam, U;
+        auto tp1 = clk::now();
         if (!sym_eig(Tc.data(), m, lam, U)) return fail(c, FD_ERR_NOT_CONVERGED, "projected eigenproblem failed");
+        auto tp2 = clk::now();
+        t_rr += secs(tp0, tp1); t_eig += secs(tp1, tp2);
         nsel = std::min(nsel_max, m);
         theta.resize(nsel);
         Xr.assign((size_t)m * nsel, 0.0);
@@ -280,6 +287,8 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             FD_TRY(S.to_host(w * w));
             for (int jj = 0; jj < w; ++jj) resid[c0 + jj] = std::sqrt(std::max(0.0, S.h_out[jj + (size_t)jj * w]));
         }
+        auto tp3 = clk::now();
+        t_res += secs(tp2, tp3);
         const double thr = tol * std::fabs(theta[0]);
         nconv = 0;
         while (nconv < std::min(nwant, nsel) && resid[nconv] <= thr) ++nconv;
@@ -351,6 +360,8 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
             FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
         }
+        auto tp4 = clk::now();
+        t_restart += secs(tp3, tp4);
         // ---- orthogonalise the new block against the basis and within itself ---------------------
         int p = (int)pick.size();
         FD_TRY(S.project_out(S.R, p, S.m));
@@ -371,8 +382,12 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             if (p == 0) break;
         }
         FD_TRY(copy_cols(c, S.R, N, S.Q + (int64_t)S.m * N, N, p, N));
+        auto tp5 = clk::now();
+        t_orth += secs(tp4, tp5);
         FD_TRY(S.apply_cols(S.m, p, b));
+        auto tp6 = clk::now();
         FD_TRY(S.extend_projection(p));
+        t_ext += secs(tp6, clk::now());
     }
 
     // ---- outputs: evecs = Q X[:, 0 : k + 1) ----------------------------------------------------------
@@ -390,6 +405,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         for (int i = 0; i < nwant; ++i) evals_host[i] = i < nout ? theta[i] : 0.0;
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
     }
+    if (getenv("FD_EIGS_TIMING"))
+        fprintf(stderr, "fd_eigs: RR setup %.3f s, small eig %.3f s, residuals %.3f s, select+restart %.3f s, orthogonalise %.3f s, apply %.3f s, extend projection %.3f s\n",
+                t_rr, t_eig, t_res, t_restart, t_orth, S.t_apply, t_ext);
     if (info) {
         info->applies = S.applies; info->restarts = S.restarts; info->converged = nconv; info->basis_cols = S.m;
         double mx = 0.0;
