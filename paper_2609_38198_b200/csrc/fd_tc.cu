@@ -200,10 +200,20 @@ __host__ __device__ constexpr uint32_t idesc_f16(int n) {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// Tuning aids (clock stamps, work-skipping switches) are compiled in only with -DFD_TC_DEBUG=1: even a never-taken
+// branch inside the exponential loop costs the hot kernel tens of percent.
+#ifndef FD_TC_DEBUG
+#define FD_TC_DEBUG 0
+#endif
+#define FD_DBG(bit) (FD_TC_DEBUG && (p.dbg & (bit)))
+#if FD_TC_DEBUG
 #define FD_TRACE(role, tile, ev)                                                                   \
     do {                                                                                          \
         if (p.trace && blockIdx.x == 0 && (tile) < 64) p.trace[((role) * 64 + (tile)) * 8 + (ev)] = clock64(); \
     } while (0)
+#else
+#define FD_TRACE(role, tile, ev) do { } while (0)
+#endif
 
 // ------------------------------------------------------------------------------------------------ shared memory map
 template <int BT, int MODE>
@@ -546,13 +556,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const uint32_t addr = tmem + lane_addr + 128u * buf;
                     // whole S row into registers first (the four loads overlap), then exponentials and in-place stores
                     uint32_t sv[4][32];
-                    if (!(p.dbg & 2)) {
+                    if (!FD_DBG(2)) {
 #pragma unroll
                     for (int qd = 0; qd < 4; ++qd) tmem_ld32(addr + 32 * qd, sv[qd]);
                     tmem_wait_ld();
                     }
                     if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 2);
-                    if (!(p.dbg & 1))
+                    if (!FD_DBG(1))
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch) {
                         uint32_t hi[8], lo[8];
