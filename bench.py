@@ -37,7 +37,7 @@ MUFU_PER_CLK_SM = 16
 FMA_PER_CLK_SM = 128
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None.
-NCU_TRAFFIC_BYTES = {"simt": None, "tc": 45.9e9 + 2.19e9}   # k_tc block mode at N = 2^20, profiles/bench_c5_n2e20_launch_list.md
+NCU_TRAFFIC_BYTES = {"simt": None, "tc": 20.15e9 + 2.18e9}   # k_tc block mode at N = 2^20, profiles/bench_c5_n2e20_launch_list.md
 
 
 def measured_peaks():
