@@ -350,7 +350,49 @@ def time_to_k_eigs(fd, dev, full=False):
         del ctx, X
         torch.cuda.empty_cache()
         res.append(rec)
+    res.append(ladder(fd, dev, full))
     return res
+
+
+def ladder(fd, dev, full=False):
+    """The (n, beta) continuation of Sec. 1 at fixed beta = 2: nested levels (first n rows of one draw), each level's solve
+    warm-started from the previous level's eigenpairs through the out-of-sample extension (fd_ladder_start), with the
+    cold-started solve of the same level beside it.  Default: 2^15 -> 2^16 -> 2^17 (k = 64, b = 32); --eigs-full: the
+    2^16 ... 2^20 ladder with k = 128, b = 64."""
+    import torch
+    import workloads
+    levels, k, b = ([1 << e for e in range(16, 21)], 128, 64) if full else ([1 << 15, 1 << 16, 1 << 17], 64, 32)
+    Xall = torch.from_numpy(workloads.torus6(levels[-1], seed=42)).to(dev)
+    m_max = (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
+    out = {"workload": f"6-torus ladder N = {levels}, k={k}, b={b}, alpha=1, beta=2.0, tol=1e-6", "levels": []}
+    prev = None
+    t_all = time.perf_counter()
+    for n in levels:
+        X = Xall[:n]
+        ctx = fd.Context(X, b_max=b, m_max=m_max)
+        t0 = time.perf_counter()
+        ctx.degree(2.0, 1.0)
+        rec = {"N": n}
+        if prev is not None:
+            pctx, plam, pU = prev
+            Q0 = ctx.ladder_start(pctx, X, pU, plam)
+            t1 = time.perf_counter()
+            lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=400, Q0=Q0, allow_not_converged=True)
+            rec.update(extend_s=t1 - t0, warm_s=time.perf_counter() - t1, warm_applies=int(info.applies),
+                       warm_converged=int(info.converged))
+            pctx.close()
+        t2 = time.perf_counter()
+        lam_c, U_c, info_c = ctx.eigs(k, b, tol=1e-6, max_applies=400, allow_not_converged=True)
+        rec.update(cold_s=time.perf_counter() - t2, cold_applies=int(info_c.applies), cold_converged=int(info_c.converged))
+        if prev is None:
+            lam, U = lam_c, U_c
+        else:
+            rec["max_eval_diff_warm_vs_cold"] = float(abs(lam - lam_c).max())
+        out["levels"].append(rec)
+        prev = (ctx, lam, U)
+    prev[0].close()
+    out["seconds"] = time.perf_counter() - t_all
+    return out
 
 
 def cpu_baseline(X, V, cfg):

@@ -81,8 +81,8 @@ fd_status fd_destroy(fd_ctx* ctx);
 
 /* Tuning / test knobs by name: "path" (FD_PATH_*), "splits" (0 = auto), "flush" (column tiles
  * between accumulator flushes of the tensor-core kernel), "tc_max_mag" (largest beta * log2(e) *
- * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "poly_exp" (share
- * of exponentials sent to the FMA pipe, 0..1), "trace" (tuning aid: the tensor-core kernel stamps
+ * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "jt_chunk" (column
+ * tiles per L2-resident chunk of the tensor-core block product), "trace" (tuning aid: the tensor-core kernel stamps
  * clock values of its first tiles into scratch), "wait_selftest" (value = limit in SM cycles: enqueues
  * a one-thread kernel whose bounded wait on a barrier that nothing completes must expire; the next
  * fd_synchronize then returns FD_ERR_TIMEOUT and the context stays usable).  fd_get_option also reports "last_path" (the
@@ -184,6 +184,18 @@ fd_status fd_beta_flow(fd_ctx* ctx, const fd_flow_opts* opts, const float* Q0_de
 fd_status fd_nystrom(fd_ctx* ctx, const float* Xnew_dev, int64_t Nnew, int64_t ldxnew,
                      const float* psi_dev, int64_t ldpsi, int32_t m, const double* lambda_host,
                      float* out_dev, int64_t ldout);
+
+/* Start basis for the next level of the (n, beta) ladder (Sec. 1: find the eigenspace on n points, extend it to a
+ * larger nested sample, re-solve there).  old_level: context over the first n_old points with its current
+ * (beta, alpha, q, d); evecs_old_dev (n_old x m, column-major) and evals_host (m) are its eigenpairs of M.
+ * new_level: context over N_new >= n_old points whose first n_old rows are the old points, after fd_degree (its d is
+ * used); Xnew_dev: the new level's points (row-major, pitch ldxnew).  Writes Q0_dev (N_new x m, pitch ldq0):
+ * Markov vectors psi = d_old^-1/2 * v on the old points, their out-of-sample extension (fd_nystrom) on the new
+ * points, all rows times d_new^1/2.  Not orthonormalised: pass it to fd_eigs / fd_beta_flow as the warm start.
+ * Synchronous. */
+fd_status fd_ladder_start(fd_ctx* old_level, fd_ctx* new_level, const float* Xnew_dev, int64_t ldxnew,
+                          const float* evecs_old_dev, int64_t ldv_old, int32_t m, const double* evals_host,
+                          float* Q0_dev, int64_t ldq0);
 
 /* Elementwise helper for the end of Sec. 2.3: out(i, c) = v(i, c) * d_i^power with the
  * context's current d (power = -0.5: Markov right eigenvectors from symmetric ones). */

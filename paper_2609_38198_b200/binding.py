@@ -25,7 +25,7 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 # Every symbol include/fd.h declares (checked by the CPU test-suite against the header).
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
-    "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree",
+    "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_ladder_start", "fd_scale_by_degree",
     "fd_apply_general_static", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
@@ -72,6 +72,9 @@ def _load() -> ctypes.CDLL:
                                  c_int64]
     lib.fd_nystrom.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int32, POINTER(c_double),
                                c_void_p, c_int64]
+    lib.fd_ladder_start.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int32, POINTER(c_double),
+                                    c_void_p, c_int64]
+    lib.fd_ladder_start.restype = c_int32
     lib.fd_scale_by_degree.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_double, c_void_p, c_int64]
     for name in ("fd_synchronize", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree", "fd_apply",
                  "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree"):
@@ -254,6 +257,16 @@ class Context:
             self._check(lib.fd_nystrom(self._h, _ptr(Xnew), Xnew.shape[0], Xnew.stride(0), _ptr(psi), _ld(psi), m, lam,
                                        _ptr(out), _ld(out)))
         return out
+
+    def ladder_start(self, old: "Context", Xnew: torch.Tensor, evecs_old: torch.Tensor, evals) -> torch.Tensor:
+        """Warm-start basis for this (new, larger) level from the eigenpairs of `old` (the level over its first rows)."""
+        m = evecs_old.shape[1]
+        lam = (c_double * m)(*[float(v) for v in evals])
+        Q0 = _colmajor(self.N, m, self.device)
+        with torch.cuda.device(self.device):
+            self._check(lib.fd_ladder_start(old._h, self._h, _ptr(Xnew), Xnew.stride(0), _ptr(evecs_old), _ld(evecs_old), m,
+                                            lam, _ptr(Q0), _ld(Q0)))
+        return Q0
 
     def scale_by_degree(self, v: torch.Tensor, power: float) -> torch.Tensor:
         out = _colmajor(self.N, v.shape[1], self.device)

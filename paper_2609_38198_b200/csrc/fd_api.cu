@@ -157,9 +157,6 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
         return tc_wait_selftest(c, (long long)v);
     } else if (!strcmp(name, "trace")) {
         c->opt_trace = (int)v;
-    } else if (!strcmp(name, "poly_exp")) {
-        if (v < 0 || v > 1) return fail(c, FD_ERR_INVALID, "poly_exp out of range");
-        c->opt_poly = v;
     } else {
         return fail(c, FD_ERR_INVALID, "unknown option %s", name);
     }
@@ -171,7 +168,6 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     if (!strcmp(name, "path")) *v = c->opt_path;
     else if (!strcmp(name, "splits")) *v = c->opt_splits;
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
-    else if (!strcmp(name, "poly_exp")) *v = c->opt_poly;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "last_path")) *v = c->last_path;
     else if (!strcmp(name, "trace_offset")) *v = (double)c->L.part;
@@ -253,7 +249,14 @@ fd_status fd_apply_general(fd_ctx* c, double beta, const float* left_dev, const 
     if (V_dev) {
         const char* v0 = (const char*)V_dev; const char* v1 = v0 + ((size_t)ldv * (b - 1) + N) * 4;
         const char* y0 = (const char*)Y_dev; const char* y1 = y0 + ((size_t)ldy * (b - 1) + Nrow) * 4;
-        if (v0 < y1 && y0 < v1) return fail(c, FD_ERR_INVALID, "V and Y overlap");
+        bool overlap = v0 < y1 && y0 < v1;
+        if (overlap && ldv == ldy) {
+            // two row ranges of one pitched panel (e.g. old rows in, new rows out, of the same basis) never touch
+            const int64_t off = ((const float*)Y_dev - (const float*)V_dev);
+            const int64_t r = ((off % ldv) + ldv) % ldv;          // first row of Y inside V's panel
+            if (r >= N && r + Nrow <= ldv) overlap = false;
+        }
+        if (overlap) return fail(c, FD_ERR_INVALID, "V and Y overlap");
     }
     ApplyArgs a{};
     a.beta = beta; a.right = right_dev; a.V = V_dev; a.ldv = ldv; a.b = b; a.prec = prec; a.rowsq = nullptr;

@@ -301,9 +301,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             for (int i = 0; i < std::min(nwant, nsel); ++i) worst = std::max(worst, resid[i]);
             if (nsel >= nwant && worst < 0.9 * best_res) { best_res = worst; since_best = 0; }
             else if (nsel >= nwant) ++since_best;
-            // the largest wanted residual has not improved by 10 % over 12 expansions and is within 30x of the target:
+            // the largest wanted residual has not improved by 10 % over 25 expansions and is within 2x of the target:
             // the operator's own rounding error is the floor; more applies do not help
-            if (since_best >= 12 && best_res <= 30.0 * thr) break;
+            if (since_best >= 25 && best_res <= 2.0 * thr) break;
         }
         if (m >= N) break;                                        // basis spans everything: nothing more to add
 

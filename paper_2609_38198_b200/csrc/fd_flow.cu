@@ -173,3 +173,27 @@ extern "C" fd_status fd_nystrom(fd_ctx* c, const float* Xnew_dev, int64_t Nnew, 
     FD_CUDA(c, cudaStreamSynchronize(c->stream));
     return FD_OK;
 }
+
+extern "C" fd_status fd_ladder_start(fd_ctx* old_level, fd_ctx* new_level, const float* Xnew_dev, int64_t ldxnew,
+                                     const float* evecs_old_dev, int64_t ldv_old, int32_t m, const double* evals_host,
+                                     float* Q0_dev, int64_t ldq0) {
+    if (!old_level || !new_level) return FD_ERR_INVALID;
+    fd_ctx* c = new_level;
+    if (!old_level->have_s || !new_level->have_s) return fail(c, FD_ERR_INVALID, "fd_ladder_start: both levels need fd_degree first");
+    const int64_t n_old = old_level->L.N, n_new = new_level->L.N;
+    if (n_new < n_old || old_level->L.D != new_level->L.D) return fail(c, FD_ERR_INVALID, "fd_ladder_start: levels are not nested");
+    if (!Xnew_dev || !evecs_old_dev || !evals_host || !Q0_dev || m < 1 || ldv_old < n_old || ldq0 < n_new || ldxnew < c->L.D)
+        return fail(c, FD_ERR_INVALID, "fd_ladder_start: bad argument");
+    // Markov vectors on the old points, written into the first n_old rows of Q0
+    FD_TRY(scale_cols_by_pow(old_level, evecs_old_dev, ldv_old, m, old_level->d(), -0.5, Q0_dev, ldq0, n_old));
+    // their extension to the points that are new at this level
+    if (n_new > n_old) {
+        fd_status st = fd_nystrom(old_level, Xnew_dev + n_old * ldxnew, n_new - n_old, ldxnew, Q0_dev, ldq0, m, evals_host,
+                                  Q0_dev + n_old, ldq0);
+        if (st != FD_OK) return fail(c, st, "fd_ladder_start: extension failed: %s", fd_last_error(old_level));
+    }
+    // back to the symmetric operator's coordinates at the new level: v = d_new^1/2 * psi
+    FD_TRY(scale_cols_by_pow(new_level, Q0_dev, ldq0, m, new_level->d(), 0.5, Q0_dev, ldq0, n_new));
+    FD_CUDA(c, cudaStreamSynchronize(c->stream));
+    return FD_OK;
+}

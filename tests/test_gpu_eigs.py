@@ -226,3 +226,30 @@ def test_nystrom_matches_oracle_and_reproduces_samples(fd, dev):
     same = ctx.nystrom(torch.from_numpy(X[:300].copy()).to(dev), psi_dev, lam_o).cpu().numpy()
     assert np.abs(same - psi_o[:300]).max() <= 5e-5 * np.abs(psi_o).max()
     ctx.close()
+
+
+def test_ladder_start_matches_oracle_and_warm_solve(fd, dev):
+    """One rung of the (n, beta) ladder: eigenpairs on the first 2500 points -> start basis on 5000 points.
+    Inputs to the extension (eigenvectors, eigenvalues) come from the oracle; the GPU and the oracle both extend them.
+    The warm-started solve on the larger level must agree with the cold one."""
+    X = workloads.torus6(5000, seed=13)
+    n_old, N, beta, alpha, k, b = 2500, 5000, 0.6, 1.0, 12, 8
+    Xo = X[:n_old]
+    lam_o, U_o, d_old = dense.eigs(Xo, beta, alpha, k)
+    q_old = dense.degree(Xo, beta, alpha)[0]
+    _, d_new, _, _, _ = dense.degree(X, beta, alpha)
+    psi_o = dense.markov_vectors(U_o, d_old)
+    ext = nystrom.extend(Xo, q_old, alpha, beta, psi_o, lam_o, X[n_old:])
+    Q0_o = np.concatenate([psi_o, ext], axis=0) * np.sqrt(d_new)[:, None]
+    old = fd.Context(torch.from_numpy(Xo.copy()).to(dev), b_max=b)
+    old.degree(beta, alpha)
+    new = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=default_m_max(k, b))
+    new.degree(beta, alpha)
+    Q0 = new.ladder_start(old, torch.from_numpy(X).to(dev), fd.to_colmajor(U_o, dev), lam_o)
+    assert np.abs(Q0.cpu().numpy() - Q0_o).max() <= 3e-5 * np.abs(Q0_o).max()
+    lam_w, U_w, info_w = new.eigs(k, b, Q0=Q0)
+    lam_c, U_c, info_c = new.eigs(k, b)
+    assert np.abs(lam_w - lam_c).max() <= 1e-6
+    check_eigs(lam_w, U_w.cpu().numpy(), X, beta, alpha, k)
+    print(f"ladder rung 2500 -> 5000: warm {info_w.applies} applies, cold {info_c.applies} applies")
+    old.close(); new.close()
