@@ -316,29 +316,41 @@ def run_gpu(args):
 
 
 def time_to_k_eigs(fd, dev, full=False):
-    """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs), and the whole
-    dyadic bandwidth flow, on the 6-torus workloads (C3: N = 2^17, b = 32, k = 64; with --eigs-full also C5: N = 2^20,
-    b = 64, k = 128).  Host wall clock around synchronous calls."""
+    """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs) on the
+    benchmark configurations at full size (C1, C2 at beta = 10 and 30, C3, C4; with --eigs-full also C5 at N = 2^20), the
+    whole dyadic bandwidth flow on C3, and the nested-level ladder.  Host wall clock around synchronous calls."""
     import torch
     import workloads
     res = []
-    cases = [("C3", 1 << 17, 64, 32)] + ([("C5", 1 << 20, 128, 64)] if full else [])
-    for name, N, k, b in cases:
-        X = torch.from_numpy(workloads.torus6(N, seed=42)).to(dev)
+    # (name, points, k, b, beta): the five benchmark configurations at their full sizes
+    cases = [("C1 circle", workloads.circle(2048), 8, 8, 200.0),
+             ("C2 2-torus", workloads.torus2(16384, seed=42), 32, 16, 10.0),
+             ("C2 2-torus", None, 32, 16, 30.0),
+             ("C3 6-torus", workloads.torus6(1 << 17, seed=42), 64, 32, 2.0),
+             ("C4 latent torus R^30", workloads.latent_torus(262144, seed=42), 32, 32, 2.0)]
+    if full:
+        cases.append(("C5 6-torus", workloads.torus6(1 << 20, seed=42), 128, 64, 2.0))
+    Xnp = None
+    for name, Xc, k, b, beta in cases:
+        if Xc is not None:
+            Xnp = Xc
+        N = Xnp.shape[0]
+        X = torch.from_numpy(Xnp).to(dev)
         m_max = (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
         ctx = fd.Context(X, b_max=b, m_max=m_max)
-        ctx.degree(2.0, 1.0)                                         # warm-up of both passes
+        ctx.degree(beta, 1.0)                                        # warm-up of both passes
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
-        ctx.degree(2.0, 1.0)
+        ctx.degree(beta, 1.0)
         t1 = time.perf_counter()
-        lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=400, allow_not_converged=True)
+        lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=600, allow_not_converged=True)
         t2 = time.perf_counter()
-        rec = {"workload": f"{name}: 6-torus N={N}, k={k}, b={b}, alpha=1, beta=2.0, tol=1e-6", "degree_s": t1 - t0,
+        rec = {"workload": f"{name}: N={N}, D={Xnp.shape[1]}, k={k}, b={b}, alpha=1, beta={beta}, tol=1e-6",
+               "path": "tc" if ctx.get_option("last_path") == 2 else "simt", "degree_s": t1 - t0,
                "eigs_s": t2 - t1, "total_s": t2 - t0, "applies": int(info.applies), "restarts": int(info.restarts),
                "converged": int(info.converged), "of": k + 1, "max_residual": float(info.max_residual),
                "seconds_in_apply": float(info.seconds_apply), "lambda_1": float(lam[1]), "lambda_k": float(lam[k])}
-        if name == "C3":
+        if name.startswith("C3"):
             t3 = time.perf_counter()
             bx, outcome, lam2, U2, recs = ctx.beta_flow(k, b, 1.0, beta_start=1.0, beta_max=1000.0, tol=1e-6, max_applies=400)
             t4 = time.perf_counter()
