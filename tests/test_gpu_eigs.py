@@ -253,3 +253,22 @@ def test_ladder_start_matches_oracle_and_warm_solve(fd, dev):
     check_eigs(lam_w, U_w.cpu().numpy(), X, beta, alpha, k)
     print(f"ladder rung 2500 -> 5000: warm {info_w.applies} applies, cold {info_c.applies} applies")
     old.close(); new.close()
+
+
+@pytest.mark.parametrize("beta_start,beta_max,expect", [(0.43, 1000.0, "LEFT_EDGE"), (0.0, 0.11, "RIGHT_EDGE")])
+def test_beta_flow_edge_outcomes_match_oracle(fd, dev, beta_start, beta_max, expect):
+    # edge rules the paper leaves open: potential already rising at the second probe / grid exhausted while falling
+    N, alpha, k = 1024, 0.5, 3
+    X = workloads.torus6_paper(N, seed=42)
+    b0 = flow.beta0(X) if beta_start <= 0 else beta_start
+    bx_o, status_o, log_o = flow.beta_flow(flow.dense_probe(X, alpha, k), N, b0, beta_max)
+    assert status_o == expect
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    bx, status, lam, U, recs = ctx.beta_flow(k, 8, alpha, beta_start=beta_start, beta_max=beta_max)
+    assert status == status_o
+    assert bx == pytest.approx(bx_o, rel=1e-6)
+    assert len(recs) == len(log_o)
+    assert ctx.get_option("beta") == pytest.approx(bx)
+    lam_o, _, _ = dense.eigs(X, bx_o, alpha, k)
+    assert np.abs(lam - lam_o).max() <= 1e-6
+    ctx.close()
