@@ -532,17 +532,19 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     ++n_grp;
                     tc_fence_after();
                     const uint32_t yaddr = tmem + lane_addr + kYCol + 64 * t;
+                    // all loads first, one wait (the S registers are free between tiles), and the accumulator is handed
+                    // back before the additions
+                    uint32_t v[BT / 16][16];
 #pragma unroll
-                    for (int c0 = 0; c0 < BT; c0 += 16) {
-                        uint32_t v[16];
-                        tmem_ld16(yaddr + c0, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) acc[(c0 + i) % BT] = fmaf(__uint_as_float(v[i]), corr, acc[(c0 + i) % BT]);
-                    }
+                    for (int c0 = 0; c0 < BT / 16; ++c0) tmem_ld16(yaddr + 16 * c0, v[c0]);
+                    tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->y_empty[t]);
+#pragma unroll
+                    for (int c0 = 0; c0 < BT / 16; ++c0)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[16 * c0 + i] = fmaf(__uint_as_float(v[c0][i]), corr, acc[16 * c0 + i]);
                     return true;
                 };
                 for (int j = 0; j < num_jt && ok; ++j) {
@@ -848,7 +850,7 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.left = a.left; p.status = status;
     p.dbg = c->opt_trace >> 1;
     p.trace = (c->opt_trace & 1) ? reinterpret_cast<long long*>(c->at<char>(L.part)) : nullptr;   // tuning aid: stamps land in the split-partials scratch
-    p.flush = c->opt_flush > 0 ? c->opt_flush : 2;
+    p.flush = c->opt_flush > 0 ? c->opt_flush : 1;
     const int grid = std::min(p.num_work, c->sm_count);
 
     if (rowsum) {
