@@ -146,6 +146,9 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "flush")) {
         if (v < 0 || v > 1 << 20) return fail(c, FD_ERR_INVALID, "flush out of range");
         c->opt_flush = (int)v;
+    } else if (!strcmp(name, "tc_variant")) {
+        if (v != 0 && v != 1) return fail(c, FD_ERR_INVALID, "tc_variant must be 0 or 1");
+        c->opt_tc_variant = (int)v;
     } else if (!strcmp(name, "jt_chunk")) {
         if (v < 0 || v > 1 << 24) return fail(c, FD_ERR_INVALID, "jt_chunk out of range");
         c->opt_jt_chunk = (int)v;

@@ -626,6 +626,313 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     }
 }
 
+// ------------------------------------------------------------------------------------------------ block-mode kernel
+// One 128-row tile per CTA.  Both warpgroups work on the SAME S tile (warpgroup h takes its columns [64 h, 64 h + 64)),
+// so all three ring buffers (3 x 128 TMEM columns) serve this one row tile and the remaining 128 columns hold a
+// double-width accumulator.  That allows the product of a K step to be issued as
+//     [Y_hh | Y_hl] += P_hi [W_hi | W_lo]      (one MMA, N = 2 BT: W_hi and W_lo tiles are adjacent in shared memory)
+//      Y_hh         += P_lo  W_hi              (one MMA, N = BT)
+// i.e. two MMAs instead of three and a wide one instead of two narrow ones (an M128 N64 K16 MMA takes ~50 clk, an
+// N128 one 64 clk).  The flush adds Y_hh + Y_hl into registers.  One product issuer, one Gram issuer.
+template <int BT, int FAST>
+struct SmemB {
+    static constexpr int kXChunk = 128 * 64;
+    static constexpr int kWHalf = BT * 128;                          // 64 j x BT columns fp16
+    static constexpr int kWBytes = (FAST ? 2 : 4) * kWHalf;           // block: [hi h0][lo h0][hi h1][lo h1]; fast: [hi h0][hi h1]
+    static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
+    static __host__ __device__ constexpr int total(int K16) {
+        return 1024 + kStages * stage_bytes(K16) + K16 * kXChunk + 1024;
+    }
+};
+
+struct BarriersB {
+    uint64_t full[kStages], empty[kStages];
+    uint64_t xfull, xempty;
+    uint64_t s_full[3];                     // S tile ready (Gram issuer -> both warpgroups)
+    uint64_t p_done[3][2];                  // warpgroup h has written its half of P in place
+    uint64_t kw_done[3];                    // product MMAs that read this buffer have completed
+    uint64_t y_full, y_empty;               // accumulator flush hand-off
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int BT, int FAST>
+__global__ void __launch_bounds__(384, 1)
+k_tcb(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUtensorMap map_xcol,
+      const __grid_constant__ CUtensorMap map_whi, const __grid_constant__ CUtensorMap map_wlo, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    using SM = SmemB<BT, FAST>;
+    constexpr int NBUF = 3;
+    constexpr uint32_t kYCol = 384;                    // accumulator: columns [384, 384 + 2 BT): Y_hh then Y_hl
+    const int K16 = p.K16;
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_base = base;
+    uint8_t* xi_base = base + kStages * SM::stage_bytes(K16);
+    BarriersB* bars = (BarriersB*)(xi_base + K16 * SM::kXChunk);
+    volatile int* abort_flag = &bars->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
+        for (int u = 0; u < 3; ++u) {
+            mbar_init(&bars->s_full[u], 1); mbar_init(&bars->kw_done[u], 1);
+            mbar_init(&bars->p_done[u][0], 4); mbar_init(&bars->p_done[u][1], 4);
+        }
+        mbar_init(&bars->y_full, 1); mbar_init(&bars->y_empty, 8);
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    // work items: (column chunk c, row tile r), c outermost, r = blockIdx.x + k * gridDim.x (see k_tc)
+    const int my_rows = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_items = my_rows * p.num_chunks;
+    const int flush = p.flush;
+#define FD_ITEM_B(w)                                                                                \
+    const int cch = (w) / my_rows;                                                                  \
+    const int item = (int)blockIdx.x + ((w) % my_rows) * (int)gridDim.x;                            \
+    const int j0 = cch * p.jt_chunk;                                                                \
+    const int num_jt = (p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk;                   \
+    (void)item; (void)cch; (void)j0
+
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(40));
+      if (warp == 8) {
+        // =============================================================== TMA producer
+        if (lane == 0) {
+            prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol); prefetch_tmap(&map_whi);
+            if (!FAST) prefetch_tmap(&map_wlo);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_B(w);
+                ok = mbar_wait(&bars->xempty, (w & 1) ^ 1, abort_flag, p.status, 1);
+                if (!ok) break;
+                mbar_expect_tx(&bars->xfull, K16 * SM::kXChunk);
+                for (int c = 0; c < K16; ++c)
+                    tma_load_2d(xi_base + c * SM::kXChunk, &map_xrow, 0, (int)(c * p.np_rows + (int64_t)item * 128), &bars->xfull);
+                for (int j = 0; j < num_jt; ++j, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(&bars->empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.status, 2);
+                    if (!ok) break;
+                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                    mbar_expect_tx(&bars->full[s], SM::stage_bytes(K16));
+                    for (int c = 0; c < K16; ++c)
+                        tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)(j0 + j) * 128), &bars->full[s]);
+                    uint8_t* wst = st + K16 * SM::kXChunk;
+                    const int x0 = (j0 + j) * 128;
+                    if (FAST) {
+                        tma_load_2d(wst, &map_whi, x0, 0, &bars->full[s]);
+                        tma_load_2d(wst + SM::kWHalf, &map_whi, x0 + 64, 0, &bars->full[s]);
+                    } else {
+                        tma_load_2d(wst, &map_whi, x0, 0, &bars->full[s]);
+                        tma_load_2d(wst + SM::kWHalf, &map_wlo, x0, 0, &bars->full[s]);
+                        tma_load_2d(wst + 2 * SM::kWHalf, &map_whi, x0 + 64, 0, &bars->full[s]);
+                        tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, x0 + 64, 0, &bars->full[s]);
+                    }
+                }
+            }
+            if (!ok) {
+                const uint32_t issued = it;
+                for (uint32_t k = (issued > (uint32_t)kStages ? issued - kStages : 0); k < issued; ++k) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&bars->full[k % kStages], (k / kStages) & 1) && clock64() - t0 < 20000000ll) {}
+                }
+            }
+        }
+      } else if (warp == 10) {
+        // =============================================================== Gram MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_g = idesc_f16(128);
+            uint32_t it = 0, g = 0;
+            bool ok = true;
+            for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_B(w);
+                ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
+                if (!ok) break;
+                for (int j = 0; j < num_jt && ok; ++j, ++it, ++g) {
+                    const int s = it % kStages, buf = g % NBUF;
+                    ok = mbar_wait(&bars->kw_done[buf], ((g / NBUF) & 1) ^ 1, abort_flag, p.status, 5);
+                    if (!ok) break;
+                    ok = mbar_wait(&bars->full[s], (it / kStages) & 1, abort_flag, p.status, 4);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t s_addr = tmem + 128u * buf;
+                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                    // small cross terms first, the large hi x hi term last (each MMA rounds at its largest addend)
+                    for (int c = 0; c < K16; ++c) {
+                        const uint64_t a = smem_desc(smem_u32(xi_base + c * SM::kXChunk), 512, 4);
+                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        mma_ss(s_addr, a, b + 2, idesc_g, c > 0);
+                        mma_ss(s_addr, a + 2, b, idesc_g, 1);
+                    }
+                    for (int c = 0; c < K16; ++c) {
+                        const uint64_t a = smem_desc(smem_u32(xi_base + c * SM::kXChunk), 512, 4);
+                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        mma_ss(s_addr, a, b, idesc_g, 1);
+                    }
+                    tc_commit(&bars->s_full[buf]);
+                }
+                if (ok) tc_commit(&bars->xempty);
+            }
+        }
+      } else if (warp == 9) {
+        // =============================================================== product MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_cat = idesc_f16(FAST ? BT : 2 * BT);
+            constexpr uint32_t idesc_y = idesc_f16(BT);
+            uint32_t it = 0, g = 0, n_grp = 0;
+            bool ok = true;
+            const uint32_t y_addr = tmem + kYCol;
+            for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_B(w);
+                for (int j = 0; j < num_jt && ok; ++j, ++it, ++g) {
+                    const int s = it % kStages, buf = g % NBUF;
+                    const uint32_t ph = (g / NBUF) & 1;
+                    const bool group_start = (j % flush) == 0;
+                    const bool group_end = ((j + 1) % flush) == 0 || j + 1 == num_jt;
+                    const uint32_t wst = smem_u32(stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk);
+                    const uint32_t p_addr = tmem + 128u * buf;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        ok = mbar_wait(&bars->p_done[buf][h], ph, abort_flag, p.status, 7);
+                        if (!ok) break;
+                        if (h == 0 && group_start && n_grp > 0) {
+                            ok = mbar_wait(&bars->y_empty, (n_grp - 1) & 1, abort_flag, p.status, 6);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        // W tiles of column half h: [W_hi | W_lo] adjacent (block) or W_hi alone (fast)
+                        const uint64_t bd = smem_desc(wst + (FAST ? 1 : 2) * h * SM::kWHalf, 1024, 2);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int ks = 4 * h + k;
+                            mma_ts(y_addr, p_addr + 16 * ks, bd + 2 * k, idesc_cat, !(group_start && ks == 0));
+                            if (!FAST) mma_ts(y_addr, p_addr + 16 * ks + 8, bd + 2 * k, idesc_y, 1);
+                        }
+                    }
+                    if (!ok) break;
+                    tc_commit(&bars->kw_done[buf]);
+                    if (group_end) { tc_commit(&bars->y_full); ++n_grp; }
+                    tc_commit(&bars->empty[s]);
+                }
+            }
+        }
+      }
+    } else {
+        // =============================================================== exponential warpgroups
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(232));
+        const int h = warp >> 2;                       // column half of every tile this warpgroup takes
+        const int wq = warp & 3;
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        const int row_in_tile = wq * 32 + lane;
+        constexpr int YC = BT / 2;                     // accumulator columns per thread: [YC h, YC h + YC)
+        uint32_t g = 0, n_grp = 0;
+        bool ok = true;
+        for (int w = 0; w < my_items && ok; ++w) {
+            FD_ITEM_B(w);
+            const int64_t row = (int64_t)item * 128 + row_in_tile;
+            float acc[YC];
+#pragma unroll
+            for (int c = 0; c < YC; ++c) acc[c] = 0.f;
+            bool pending = false;
+            // Flush: adds the TMEM accumulator into registers and hands it back.  The tensor core accumulates with
+            // round-toward-zero; n same-sign additions lose n / 4 ulp on average (measured 2.85e-8 each vs 2^-25), which the
+            // flush adds back: Y_hh receives two additions per K step (one in fast mode), Y_hl one.
+            auto do_flush = [&](int tiles_in_group) -> bool {
+                const float c_hh = 1.0f + (float)(tiles_in_group * 8 * (FAST ? 1 : 2)) * 2.98023224e-8f;
+                const float c_hl = 1.0f + (float)(tiles_in_group * 8) * 2.98023224e-8f;
+                if (!mbar_wait(&bars->y_full, n_grp & 1, abort_flag, p.status, 10)) return false;
+                ++n_grp;
+                tc_fence_after();
+                const uint32_t yaddr = tmem + lane_addr + kYCol + YC * h;
+                constexpr int NL = YC >= 16 ? YC / 16 : 1;
+                uint32_t vh[NL][16], vl[NL][16];
+#pragma unroll
+                for (int c0 = 0; c0 < NL; ++c0) tmem_ld16(yaddr + 16 * c0, vh[c0]);
+                if (!FAST) {
+#pragma unroll
+                    for (int c0 = 0; c0 < NL; ++c0) tmem_ld16(yaddr + BT + 16 * c0, vl[c0]);
+                }
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->y_empty);
+#pragma unroll
+                for (int c = 0; c < YC; ++c) {
+                    acc[c] = fmaf(__uint_as_float(vh[c / 16][c % 16]), c_hh, acc[c]);
+                    if (!FAST) acc[c] = fmaf(__uint_as_float(vl[c / 16][c % 16]), c_hl, acc[c]);
+                }
+                return true;
+            };
+            for (int j = 0; j < num_jt && ok; ++j, ++g) {
+                const int buf = g % NBUF;
+                ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 9);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t addr = tmem + lane_addr + 128u * buf + 64u * h;
+                uint32_t sv[2][32];
+                tmem_ld32(addr, sv[0]);
+                tmem_ld32(addr + 32, sv[1]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t hi[8], lo[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float p0 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i]));
+                        const float p1 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i + 1]));
+                        if (!FAST) {
+                            const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
+                            const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
+                            hi[i] = pack_f16x2(h0, h1);
+                            lo[i] = pack_f16x2(p0 - h0, p1 - h1);
+                        } else {
+                            hi[i] = pack_f16x2(p0, p1);
+                        }
+                    }
+                    tmem_st8(addr + 16 * ch, hi);
+                    if (!FAST) tmem_st8(addr + 16 * ch + 8, lo);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->p_done[buf][h]);
+                if (pending) { ok = do_flush(flush); pending = false; if (!ok) break; }
+                if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
+                    if (j + 1 == num_jt) { ok = do_flush(j % flush + 1); if (!ok) break; }
+                    else pending = true;
+                }
+            }
+            if (ok && row < p.Nrow) {
+                const float l = p.left ? p.left[row] : 1.0f;
+#pragma unroll
+                for (int c = 0; c < YC; ++c) {
+                    const int col = YC * h + c;
+                    if (col < p.b) {
+                        float* o = p.Y + row + (int64_t)col * p.ldy;
+                        const float v = acc[c] * l * p.colscale_inv[col];
+                        *o = cch == 0 ? v : *o + v;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
 // Exercises the bounded-wait path without any fault: one thread waits on a barrier that nothing will ever complete,
 // with a short limit; the wait gives up, records its code in the status word and the kernel returns normally.
 __global__ void k_wait_selftest(unsigned int* status, long long limit_cycles) {
@@ -793,6 +1100,21 @@ fd_status launch_tc(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, con
     return FD_OK;
 }
 
+template <int BT, int FAST>
+fd_status launch_tcb(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, const CUtensorMap& mh, const CUtensorMap& ml,
+                     const TcParams& p, int grid) {
+    const int smem = SmemB<BT, FAST>::total(p.K16);
+    if (smem > 227 * 1024) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core kernel needs %d B of shared memory", smem);
+    static bool configured = false;
+    if (!configured) {
+        FD_CUDA(c, cudaFuncSetAttribute(k_tcb<BT, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        configured = true;
+    }
+    k_tcb<BT, FAST><<<grid, 384, smem, c->stream>>>(mr, mc, mh, ml, p);
+    FD_LAUNCH_CHECK(c, "k_tcb");
+    return FD_OK;
+}
+
 }  // namespace
 
 bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
@@ -878,9 +1200,16 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
                 !make_map_2d(&ml, wt_lo, (uint64_t)NP, (uint64_t)BT, (uint64_t)NP * 2, 64, BT, CU_TENSOR_MAP_SWIZZLE_128B))
                 return fail(c, FD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the block operands");
             p.b = bc; p.colscale_inv = inv; p.Y = a.Y + (int64_t)c0 * a.ldy; p.ldy = a.ldy;
+            TcParams pb = p;                       // one-row-tile variant: 128-row work items
+            pb.num_work = (int)ceil_div(a.Nrow, 128);
+            const int grid_b = std::min(pb.num_work, c->sm_count);
+            const bool one_tile = c->opt_tc_variant != 1;
 #define FD_TC_CASE(B)                                                                              \
     case B:                                                                                        \
-        if (fast) FD_TRY((launch_tc<B, kModeFast>(c, mr, mc, mh, ml, p, grid)));                   \
+        if (one_tile) {                                                                            \
+            if (fast) FD_TRY((launch_tcb<B, 1>(c, mr, mc, mh, ml, pb, grid_b)));                   \
+            else FD_TRY((launch_tcb<B, 0>(c, mr, mc, mh, ml, pb, grid_b)));                        \
+        } else if (fast) FD_TRY((launch_tc<B, kModeFast>(c, mr, mc, mh, ml, p, grid)));            \
         else FD_TRY((launch_tc<B, kModeBlock>(c, mr, mc, mh, ml, p, grid)));                       \
         break;
             switch (BT) { FD_TC_CASE(16) FD_TC_CASE(32) FD_TC_CASE(64) }
