@@ -31,7 +31,7 @@ import numpy as np  # noqa: E402
 METRIC = "kernel-apply pair-columns per second (degree passes + block product, one step)"
 UNIT = "pair*cols/s"
 
-# Peaks for the roofline: MUFU 16 ex2/clk/SM, FMA pipe 128 FFMA/clk/SM, 148 SMs.
+# Nominal unit counts for the roofline: MUFU 16 ex2/clk/SM, FMA pipe 128 FFMA/clk/SM, 148 SMs.
 SM_COUNT = 148
 MUFU_PER_CLK_SM = 16
 FMA_PER_CLK_SM = 128

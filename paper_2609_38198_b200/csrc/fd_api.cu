@@ -37,7 +37,9 @@ Layout make_layout(int64_t N, int32_t D, int32_t b_max, int32_t m_max) {
     Layout L;
     L.N = N; L.D = D; L.b_max = b_max; L.m_max = m_max;
     L.DP = (int32_t)round_up(D, 4);
-    L.BP = (int32_t)round_up(b_max, 16);
+    // block-width-dependent buffers are sized by the widest column tile a kernel can launch for b <= b_max
+    // (16, 32 or a multiple of 64), not by b_max itself: both kernel families pad a chunk of 33..64 columns to 64
+    L.BP = b_max <= 16 ? 16 : b_max <= 32 ? 32 : (int32_t)round_up(b_max, 64);
     L.NP = round_up(N, kTileM * kRowTilesPerCta);
     L.K16 = (int32_t)ceil_div(D + 4, 16);
     size_t cur = 0;
@@ -158,8 +160,6 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "wait_selftest")) {
         if (!(v >= 1000) || v > 4e9) return fail(c, FD_ERR_INVALID, "wait_selftest: limit in cycles, 1e3..4e9");
         return tc_wait_selftest(c, (long long)v);
-    } else if (!strcmp(name, "trace")) {
-        c->opt_trace = (int)v;
     } else {
         return fail(c, FD_ERR_INVALID, "unknown option %s", name);
     }
@@ -173,7 +173,6 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "last_path")) *v = c->last_path;
-    else if (!strcmp(name, "trace_offset")) *v = (double)c->L.part;
     else if (!strcmp(name, "mean_sq")) *v = c->mean_sq;
     else if (!strcmp(name, "max_sq")) *v = c->max_sq;
     else if (!strcmp(name, "beta")) *v = c->beta;

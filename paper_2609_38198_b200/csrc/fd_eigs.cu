@@ -405,9 +405,12 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         for (int i = 0; i < nwant; ++i) evals_host[i] = i < nout ? theta[i] : 0.0;
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
     }
-    if (getenv("FD_EIGS_TIMING"))
-        fprintf(stderr, "fd_eigs: RR setup %.3f s, small eig %.3f s, residuals %.3f s, select+restart %.3f s, orthogonalise %.3f s, apply %.3f s, extend projection %.3f s\n",
-                t_rr, t_eig, t_res, t_restart, t_orth, S.t_apply, t_ext);
+#ifdef FD_EIGS_TIMING
+    fprintf(stderr, "fd_eigs: RR setup %.3f s, small eig %.3f s, residuals %.3f s, select+restart %.3f s, orthogonalise %.3f s, apply %.3f s, extend projection %.3f s\n",
+            t_rr, t_eig, t_res, t_restart, t_orth, S.t_apply, t_ext);
+#else
+    (void)t_rr; (void)t_eig; (void)t_res; (void)t_restart; (void)t_orth; (void)t_ext;
+#endif
     if (info) {
         info->applies = S.applies; info->restarts = S.restarts; info->converged = nconv; info->basis_cols = S.m;
         double mx = 0.0;

@@ -248,6 +248,7 @@ fd_status apply_simt(fd_ctx* c, const ApplyArgs& a) {
     for (int c0 = 0; c0 < a.b; c0 += 64) {
         const int bc = a.b - c0 < 64 ? a.b - c0 : 64;
         const int BT = pick_bt(bc);
+        if (BT > L.BP) return fail(c, FD_ERR_WORKSPACE, "column tile %d wider than the provisioned block buffers (%d)", BT, L.BP);
         dim3 pg((unsigned)ceil_div(N, 32), (unsigned)ceil_div(BT, 32));
         k_pack_w<<<pg, dim3(32, 8), 0, c->stream>>>(a.V, a.ldv, a.right, N, c0, bc, BT, wp);
         FD_LAUNCH_CHECK(c, "k_pack_w");

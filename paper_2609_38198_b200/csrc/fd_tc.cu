@@ -1090,11 +1090,8 @@ fd_status launch_tc(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, con
                     const TcParams& p, int grid) {
     const int smem = Smem<BT, MODE>::total(p.K16);
     if (smem > 227 * 1024) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core kernel needs %d B of shared memory", smem);
-    static bool configured = false;
-    if (!configured) {
-        FD_CUDA(c, cudaFuncSetAttribute(k_tc<BT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        configured = true;
-    }
+    // the attribute is per device: set it on every launch (cheap) rather than remembering one device
+    FD_CUDA(c, cudaFuncSetAttribute(k_tc<BT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     k_tc<BT, MODE><<<grid, kThreads, smem, c->stream>>>(mr, mc, mh, ml, p);
     FD_LAUNCH_CHECK(c, "k_tc");
     return FD_OK;
@@ -1105,11 +1102,7 @@ fd_status launch_tcb(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, co
                      const TcParams& p, int grid) {
     const int smem = SmemB<BT, FAST>::total(p.K16);
     if (smem > 227 * 1024) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core kernel needs %d B of shared memory", smem);
-    static bool configured = false;
-    if (!configured) {
-        FD_CUDA(c, cudaFuncSetAttribute(k_tcb<BT, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        configured = true;
-    }
+    FD_CUDA(c, cudaFuncSetAttribute(k_tcb<BT, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     k_tcb<BT, FAST><<<grid, 384, smem, c->stream>>>(mr, mc, mh, ml, p);
     FD_LAUNCH_CHECK(c, "k_tcb");
     return FD_OK;
@@ -1121,6 +1114,7 @@ bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
     const Layout& L = c->L;
     if (!c->centered) return false;
     if (L.K16 > 4) return false;                                   // D <= 60
+    if ((int64_t)L.K16 * L.NP >= ((int64_t)1 << 31)) return false;    // TMA row coordinates are 32-bit
     if (a.Nrow > L.N) return false;
     // The decision depends only on the data set, the bandwidth and the precision mode -- never on the kind of pass --
     // so the degree passes and the block products of one operator always run on the same kernel family (their
@@ -1188,6 +1182,7 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
         for (int c0 = 0; c0 < a.b; c0 += 64) {
             const int bc = std::min(64, a.b - c0);
             const int BT = bc <= 16 ? 16 : bc <= 32 ? 32 : 64;
+            if (BT > L.BP) return fail(c, FD_ERR_WORKSPACE, "column tile %d wider than the provisioned block buffers (%d)", BT, L.BP);
             const int cm_blocks = (int)std::min<int64_t>(256, ceil_div(N, 1024));
             k_colmax_partial<<<dim3(cm_blocks, bc), 256, 0, c->stream>>>(a.V, a.ldv, a.right, N, c0, bc, part);
             FD_LAUNCH_CHECK(c, "k_colmax_partial");

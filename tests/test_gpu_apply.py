@@ -88,7 +88,7 @@ def test_tail_sizes(fd, dev, N):
     run_case(fd, dev, workloads.gaussian_cloud(N, 3, seed=N), 0.7, 1.0, 8 if N > 1 else 1, fd.FD_PATH_SIMT)
 
 
-@pytest.mark.parametrize("b", [1, 3, 8, 16, 33, 64, 70, 130])
+@pytest.mark.parametrize("b", [1, 3, 8, 16, 33, 40, 48, 64, 70, 130])
 def test_block_widths(fd, dev, b):
     run_case(fd, dev, workloads.torus6(700, seed=b), 1.0, 1.0, b, fd.FD_PATH_SIMT)
 

@@ -67,7 +67,7 @@ def test_row_and_column_tails(fd, dev, N):
     tc_case(fd, dev, workloads.torus6(N, seed=N), 2.0, 1.0, 64 if N > 1 else 1)
 
 
-@pytest.mark.parametrize("b", [1, 8, 16, 24, 32, 64, 70, 128])
+@pytest.mark.parametrize("b", [1, 8, 16, 24, 32, 40, 48, 64, 70, 128])
 def test_block_widths(fd, dev, b):
     tc_case(fd, dev, workloads.torus6(900, seed=b), 1.0, 1.0, b)
 

@@ -354,3 +354,39 @@ def test_t6_continuum_clusters_soft():
     lam, _, _ = dense.eigs(X, beta, 1.0, 12)
     r1 = ive(1, 2 * beta) / ive(0, 2 * beta)
     assert abs(np.mean(lam[1:13]) / r1 - 1.0) < 0.15
+
+
+# ------------------------------------------------------------------ the checker behind every angle gate
+@pytest.mark.parametrize("t", [1e-6, 1e-3, 0.3, 1.2])
+def test_principal_angles_known_single_angle(t):
+    # span{e1} against span{cos t e1 + sin t e2}: the one principal angle is t (textbook definition)
+    n = 50
+    A = np.zeros((n, 1)); A[0, 0] = 1.0
+    B = np.zeros((n, 1)); B[0, 0] = np.cos(t); B[1, 0] = np.sin(t)
+    ang = dense.principal_angles(A, B)
+    assert ang.shape == (1,)
+    assert ang[0] == pytest.approx(t, rel=1e-9, abs=1e-15)
+    # symmetric in its arguments, and insensitive to column scaling and sign
+    assert dense.principal_angles(B, A)[0] == pytest.approx(t, rel=1e-9, abs=1e-15)
+    assert dense.principal_angles(-3.0 * A, 0.25 * B)[0] == pytest.approx(t, rel=1e-9, abs=1e-15)
+
+
+def test_principal_angles_two_distinct_angles_and_nonorthonormal_columns():
+    # planes span{e1, e2} and span{c1 e1 + s1 e3, c2 e2 + s2 e4}: principal angles are exactly (t1, t2), ascending
+    n, t1, t2 = 12, 2e-4, 0.7
+    A = np.zeros((n, 2)); A[0, 0] = 1.0; A[1, 1] = 1.0
+    B = np.zeros((n, 2))
+    B[0, 0] = np.cos(t1); B[2, 0] = np.sin(t1)
+    B[1, 1] = np.cos(t2); B[3, 1] = np.sin(t2)
+    ang = dense.principal_angles(A, B)
+    assert np.allclose(ang, [t1, t2], rtol=1e-9, atol=1e-15)
+    # the same two planes given by skewed, unnormalised bases and after a common rotation of the ambient space
+    rng = np.random.default_rng(7)
+    Ta = np.array([[2.0, 1.5], [0.3, -0.7]]); Tb = np.array([[0.1, 4.0], [1.0, 1.0]])
+    Qrot, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    ang2 = dense.principal_angles(Qrot @ (A @ Ta), Qrot @ (B @ Tb))
+    assert np.allclose(ang2, [t1, t2], rtol=1e-7, atol=1e-13)
+    # identical spans: zero; orthogonal spans: pi / 2
+    assert dense.principal_angles(A, A @ Ta).max() < 1e-12
+    C = np.zeros((n, 2)); C[4, 0] = 1.0; C[5, 1] = 1.0
+    assert np.allclose(dense.principal_angles(A, C), [np.pi / 2, np.pi / 2])

@@ -4,8 +4,10 @@ A plug-in that is handed only input and output buffers, or code that runs where 
 forbids allocation, cannot give the library a workspace.  fd_apply_general_static keeps its
 scratch in the library's own fixed device array instead.  This test calls it through the C ABI
 twice in a row (the array is shared and keeps the previous call's contents, so the second call
-must not be disturbed by the first) and checks both results against the ordinary entry point
-fd_apply_general, at the tolerance the other parity tests use for the block product.  It lives
+must not be disturbed by the first) and checks both results against the float64 oracle
+(the dense definition written out; the sizes here are small enough for it) and against the
+ordinary entry point fd_apply_general, at the tolerance the other parity tests use for the block
+product.  It lives
 in a file that pytest collects last so that a failure here cannot hide any other test, and it
 passes both alone in a fresh process and after the rest of the suite.
 """
@@ -14,6 +16,7 @@ import pytest
 import torch
 
 import workloads
+from oracle import dense
 
 pytestmark = pytest.mark.gpu
 
@@ -34,6 +37,11 @@ def relF(a, b):
     return float((a - b).norm() / b.norm())
 
 
+def relF_oracle(Y, Yo):
+    Yn = Y.cpu().numpy().astype(np.float64)
+    return float(np.linalg.norm(Yn - Yo) / np.linalg.norm(Yo))
+
+
 def test_static_scratch_entry_point_matches_workspace_entry_point(fd):
     dev = torch.device("cuda:0")
     rng = np.random.default_rng(3)
@@ -41,10 +49,17 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(fd):
     for X, beta, b in cases:
         N = X.shape[0]
         Xd = torch.from_numpy(X).to(dev)
-        l = torch.from_numpy(rng.uniform(0.5, 2.0, N).astype(np.float32)).to(dev)
-        r = torch.from_numpy(rng.uniform(0.5, 2.0, N).astype(np.float32)).to(dev)
-        V1 = fd.to_colmajor(workloads.block(N, b, seed=5), dev)
-        V2 = fd.to_colmajor(workloads.block(N, b, seed=6), dev)
+        lh = rng.uniform(0.5, 2.0, N).astype(np.float32)
+        rh = rng.uniform(0.5, 2.0, N).astype(np.float32)
+        l = torch.from_numpy(lh).to(dev)
+        r = torch.from_numpy(rh).to(dev)
+        V1h, V2h = workloads.block(N, b, seed=5), workloads.block(N, b, seed=6)
+        V1 = fd.to_colmajor(V1h, dev)
+        V2 = fd.to_colmajor(V2h, dev)
+        # float64 oracle: Y = diag(l) K diag(r) V with K materialised
+        O1 = dense.apply_general(X, beta, V1h, left=lh, right=rh)
+        O2 = dense.apply_general(X, beta, V2h, left=lh, right=rh)
+        O3 = dense.apply_general(X, beta, V1h)
         # reference results from the existing entry point (caller-provided workspace, same kernel family)
         ctx = fd.Context(Xd, b_max=b)
         ctx.set_option("path", fd.FD_PATH_SIMT)
@@ -60,6 +75,8 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(fd):
         fd.fd_apply_general_static(Xd, beta, V2, left=l, right=r, out=Y2)
         torch.cuda.synchronize(dev)
         assert fd.fd_launch_count() > launches
+        assert relF_oracle(Y1, O1) <= TOL_APPLY
+        assert relF_oracle(Y2, O2) <= TOL_APPLY
         assert relF(Y1, R1) <= TOL_APPLY
         assert relF(Y2, R2) <= TOL_APPLY
         # optional scalings absent
@@ -68,6 +85,7 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(fd):
         ctx.set_option("path", fd.FD_PATH_SIMT)
         R3 = ctx.apply_general(beta, V1)
         ctx.synchronize()
+        assert relF_oracle(Y3, O3) <= TOL_APPLY
         assert relF(Y3, R3) <= TOL_APPLY
         ctx.close()
 
