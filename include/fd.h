@@ -85,7 +85,9 @@ fd_status fd_destroy(fd_ctx* ctx);
  * tiles per L2-resident chunk of the tensor-core block product), "wait_selftest" (value = limit in SM cycles: enqueues
  * a one-thread kernel whose bounded wait on a barrier that nothing completes must expire; the next
  * fd_synchronize then returns FD_ERR_TIMEOUT and the context stays usable).  fd_get_option also reports "last_path" (the
- * family that served the latest pass), "beta", "mean_sq", "max_sq".  Unknown name -> FD_ERR_INVALID. */
+ * family that served the latest pass), "beta", "mean_sq", "max_sq" and "tc_cycles" (SM cycles the first CTA of the most
+ * recent reduced-precision tensor-core block product spent on its work items; synchronises; with the kernel's wall time it
+ * gives the SM clock the kernel actually ran at).  Unknown name -> FD_ERR_INVALID. */
 fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
 fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);
 

@@ -148,9 +148,6 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "flush")) {
         if (v < 0 || v > 1 << 20) return fail(c, FD_ERR_INVALID, "flush out of range");
         c->opt_flush = (int)v;
-    } else if (!strcmp(name, "tc_variant")) {
-        if (v != 0 && v != 1) return fail(c, FD_ERR_INVALID, "tc_variant must be 0 or 1");
-        c->opt_tc_variant = (int)v;
     } else if (!strcmp(name, "jt_chunk")) {
         if (v < 0 || v > 1 << 24) return fail(c, FD_ERR_INVALID, "jt_chunk out of range");
         c->opt_jt_chunk = (int)v;
@@ -173,6 +170,13 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "last_path")) *v = c->last_path;
+    else if (!strcmp(name, "tc_cycles")) {
+        // SM cycles the first CTA of the most recent tensor-core block product spent (synchronises)
+        long long cyc = 0;
+        if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+            cudaMemcpy(&cyc, c->at<unsigned int>(c->L.status) + 2, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return FD_ERR_CUDA;
+        *v = (double)cyc;
+    }
     else if (!strcmp(name, "mean_sq")) *v = c->mean_sq;
     else if (!strcmp(name, "max_sq")) *v = c->max_sq;
     else if (!strcmp(name, "beta")) *v = c->beta;

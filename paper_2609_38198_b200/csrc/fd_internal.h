@@ -54,10 +54,8 @@ struct fd_ctx {
     int opt_path = FD_PATH_AUTO;
     int opt_splits = 0;
     int opt_flush = 0;
-    int opt_tc_variant = 0;          // block product on the tensor-core path: 0 = one row tile per CTA (k_tcb), 1 = two (k_tc)
     int opt_jt_chunk = 0;            // column tiles per L2-resident chunk of the tensor-core block product (0 = default)
     int last_path = 0;               // kernel family that served the most recent quadratic pass (FD_PATH_SIMT / FD_PATH_TC)
-    int opt_trace = 0;               // tensor-core kernel writes clock stamps of its first tiles into the partials scratch
     double opt_tc_max_mag = 72.0;    // largest beta' * max|x - mu|^2 the Gram-form kernel is trusted with in fp32 mode
     std::string err;
 

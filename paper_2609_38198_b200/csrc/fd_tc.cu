@@ -28,199 +28,20 @@
 #include <algorithm>
 #include <cmath>
 
-#include "fd_internal.h"
+#include "fd_tc_common.h"
 
 namespace fd {
 
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kThreads = 384;                // warps 0-3 / 4-7: exponential warpgroups; warps 8-11: TMA, MMA, 2 idle
-constexpr int kBias = 15;                    // P' = 2^15 P keeps fp16 hi/lo of P out of the denormal range
-constexpr uint32_t kTmemCols = 512;
-constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any legitimate wait
-
-enum Mode { kModeBlock = 0, kModeFast = 1, kModeRowsum = 2 };
-
-struct TcParams {
-    int64_t Nrow, N;             // valid rows / columns
-    int num_work;                // row-pair tiles (256 rows each)
-    int num_jt;                  // column tiles
-    int jt_chunk, num_chunks;    // the column range is swept in chunks small enough for L2 (block mode); all CTAs work on one chunk at a time
-    int64_t np_rows;             // padded row count of the operand arrays (row index of K slab c = c * np + p)
-    int64_t np_cols;
-    int K16;
-    int b;                       // real block columns to store
-    int flush;                   // column tiles per accumulator flush
-    const float* left;           // may be null
-    const float* colscale_inv;   // per column: 2^-bias / colscale
-    float* Y; int64_t ldy;
-    float* q; double* rowsq;     // row-sum outputs
-    unsigned int* status;
-    int dbg;                     // tuning aid: bit 0 = warpgroups skip exponentials and stores, bit 1 = skip the S loads too
-    long long* trace;            // optional: clock64 stamps of CTA 0's first tiles (tuning aid), [4 roles][64 tiles][8 events]
-};
-
-// ------------------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: returns false (and raises the abort flag) when the limit is hit or another role aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, int code,
-                                          long long limit = kWaitCycles) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    int spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        __nanosleep(40);            // back off: many warps polling shared memory slow the MMA issuer down
-        if ((++spins & 63) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) {
-                *abort_flag = 1;
-                atomicCAS(status, 0u, (unsigned)(0x100 | code));
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(addr) : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(addr) : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&v)[8]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-        ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ float ex2f(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-// K-major shared-memory operand descriptor (sm_100 format): start address, stride between 8-row groups,
-// swizzle mode (2 = 128 B rows, 4 = 64 B rows).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
-    d |= (uint64_t)(sbo_bytes >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)layout << 61;
-    return d;
-}
-// Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128.
-__host__ __device__ constexpr uint32_t idesc_f16(int n) {
-    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-// Tuning aids (clock stamps, work-skipping switches) are compiled in only with -DFD_TC_DEBUG=1: even a never-taken
-// branch inside the exponential loop costs the hot kernel tens of percent.
-#ifndef FD_TC_DEBUG
-#define FD_TC_DEBUG 0
-#endif
-#define FD_DBG(bit) (FD_TC_DEBUG && (p.dbg & (bit)))
-#if FD_TC_DEBUG
-#define FD_TRACE(role, tile, ev)                                                                   \
-    do {                                                                                          \
-        if (p.trace && blockIdx.x == 0 && (tile) < 64) p.trace[((role) * 64 + (tile)) * 8 + (ev)] = clock64(); \
-    } while (0)
-#else
-#define FD_TRACE(role, tile, ev) do { } while (0)
-#endif
+using namespace tc;
 
 // ------------------------------------------------------------------------------------------------ shared memory map
 template <int BT, int MODE>
 struct Smem {
     static constexpr int kXChunk = 128 * 64;                       // one K slab (hi|lo) of 128 points: 8 KB
     static constexpr int kWHalf = (MODE == kModeRowsum) ? 0 : BT * 128;   // 64 j x BT columns fp16
-    static constexpr int kWBytes = (MODE == kModeRowsum) ? 0 : (MODE == kModeFast ? 2 : 4) * kWHalf;
+    static constexpr int kWBytes = (MODE == kModeRowsum) ? 0 : 4 * kWHalf;   // [W_hi j-half 0][W_hi j-half 1][W_lo 0][W_lo 1]
     static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
     static __host__ __device__ constexpr int total(int K16) {
         return 1024 /*align slack*/ + kStages * stage_bytes(K16) + 2 * K16 * kXChunk + 1024 /*barriers*/;
@@ -309,7 +130,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         // =============================================================== TMA producer (one thread)
         if (lane == 0) {
             prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol);
-            if (MODE != kModeRowsum) { prefetch_tmap(&map_whi); if (MODE == kModeBlock) prefetch_tmap(&map_wlo); }
+            if (MODE != kModeRowsum) { prefetch_tmap(&map_whi); prefetch_tmap(&map_wlo); }
             uint32_t it = 0;
             bool ok = true;
             for (int w = 0; w < my_items && ok; ++w) {
@@ -333,10 +154,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         uint8_t* wst = st + K16 * SM::kXChunk;
                         tma_load_2d(wst, &map_whi, (j0 + j) * 128, 0, &bars->full[s]);
                         tma_load_2d(wst + SM::kWHalf, &map_whi, (j0 + j) * 128 + 64, 0, &bars->full[s]);
-                        if (MODE == kModeBlock) {
-                            tma_load_2d(wst + 2 * SM::kWHalf, &map_wlo, (j0 + j) * 128, 0, &bars->full[s]);
-                            tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, (j0 + j) * 128 + 64, 0, &bars->full[s]);
-                        }
+                        tma_load_2d(wst + 2 * SM::kWHalf, &map_wlo, (j0 + j) * 128, 0, &bars->full[s]);
+                        tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, (j0 + j) * 128 + 64, 0, &bars->full[s]);
                     }
                 }
             }
@@ -366,7 +185,6 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const int buf = g % NBUF;
                     const uint32_t itj = it0 + (uint32_t)(n >> 1);
                     const int s = itj % kStages;
-                    if (w == 0) FD_TRACE(3, n, 0);
                     if (g >= (uint32_t)NBUF) {
                         // the tile that used this buffer last (NBUF tiles ago, possibly of the other row tile) must be finished
                         const uint32_t gp = g - NBUF;
@@ -374,7 +192,6 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         ok = mbar_wait(fb, (gp / kRingPeriod) & 1, abort_flag, p.status, 5);
                         if (!ok) break;
                     }
-                    if (w == 0) FD_TRACE(3, n, 1);
                     if ((n & 1) == 0) {
                         ok = mbar_wait(&bars->full[s], (itj / kStages) & 1, abort_flag, p.status, 4);
                         if (!ok) break;
@@ -397,7 +214,6 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         mma_ss(s_addr, a, b, idesc_g, 1);
                     }
                     tc_commit(&bars->s_full[buf][n & 1]);
-                    if (w == 0) FD_TRACE(3, n, 2);
                     if (MODE == kModeRowsum && (n & 1)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
                 }
                 if (ok) tc_commit(&bars->xempty);                  // the row operand tiles may be replaced
@@ -416,21 +232,21 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             const uint32_t y_addr = tmem + kYCol + 64 * t;
             for (int w = 0; w < my_items && ok; ++w) {
                 FD_ITEM_GEOMETRY(w);
+                int in_group = 0;                                  // tiles accumulated in the current group (no division in the hot loop)
                 for (int j = 0; j < num_jt && ok; ++j) {
                     const uint32_t g = gn0 + 2u * (uint32_t)j + (uint32_t)t;
                     const int buf = g % NBUF;
                     const int s = (it0 + (uint32_t)j) % kStages;
-                    if (w == 0) FD_TRACE(0, 2 * j + t, 0);
                     ok = mbar_wait(&bars->p_half[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 7);
                     if (!ok) break;
-                    const bool group_start = (j % flush) == 0;
-                    const bool group_end = ((j + 1) % flush) == 0 || j + 1 == num_jt;
+                    const bool group_start = in_group == 0;
+                    const bool group_end = in_group + 1 == flush || j + 1 == num_jt;
+                    in_group = group_end ? 0 : in_group + 1;
                     if (group_start && n_grp > 0) {
                         ok = mbar_wait(&bars->y_empty[t], (n_grp - 1) & 1, abort_flag, p.status, 6);
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    if (w == 0) FD_TRACE(0, 2 * j + t, 1);
                     // Y_t += P W : 8 K steps of 16 columns j; K step ks reads P_hi at S-buffer columns [16 ks, 16 ks + 8)
                     // and P_lo at [16 ks + 8, 16 ks + 16) (the warpgroup wrote them in place over S).  The first four K steps
                     // start as soon as the first half of P is written, the rest once the tile is complete.
@@ -448,17 +264,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         const uint32_t off = (uint32_t)(((ks >> 2) * SM::kWHalf + (ks & 3) * 32) >> 4);
                         const uint32_t a_hi = p_addr + 16 * ks;
                         mma_ts(y_addr, a_hi, bd_hi + off, idesc_y, !(group_start && ks == 0));
-                        if (MODE == kModeBlock) {
-                            mma_ts(y_addr, a_hi + 8, bd_hi + off, idesc_y, 1);
-                            mma_ts(y_addr, a_hi, bd_lo + off, idesc_y, 1);
-                        }
+                        mma_ts(y_addr, a_hi + 8, bd_hi + off, idesc_y, 1);
+                        mma_ts(y_addr, a_hi, bd_lo + off, idesc_y, 1);
                     }
                     if (!ok) break;
-                    if (w == 0) FD_TRACE(0, 2 * j + t, 2);
                     tc_commit(&bars->kw_done[buf][t]);
                     if (group_end) { tc_commit(&bars->y_full[t]); ++n_grp; }
                     tc_commit(&bars->empty[s]);
-                    if (w == 0) FD_TRACE(0, 2 * j + t, 3);
                 }
                 it0 += (uint32_t)num_jt;
                 gn0 += (uint32_t)tiles_per_item;
@@ -527,7 +339,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 // flush adds that expected loss back (one FMA instead of one add), which removes the common scale error of
                 // M V that would otherwise shift every eigenvalue by ~7e-7 per column tile in the group.
                 auto do_flush = [&](int tiles_in_group) -> bool {
-                    const float corr = 1.0f + (float)(tiles_in_group * 8 * (MODE == kModeBlock ? 3 : 1)) * 2.98023224e-8f;
+                    const float corr = 1.0f + (float)(tiles_in_group * 8 * 3) * 2.98023224e-8f;
                     if (!mbar_wait(&bars->y_full[t], n_grp & 1, abort_flag, p.status, 10)) return false;
                     ++n_grp;
                     tc_fence_after();
@@ -547,24 +359,19 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         for (int i = 0; i < 16; ++i) acc[16 * c0 + i] = fmaf(__uint_as_float(v[c0][i]), corr, acc[16 * c0 + i]);
                     return true;
                 };
+                int in_group = 0;
                 for (int j = 0; j < num_jt && ok; ++j) {
                     const uint32_t g = gn0 + 2u * j + t;
                     const int buf = g % NBUF;
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 0);
                     ok = mbar_wait(&bars->s_full[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 9);
                     if (!ok) break;
                     tc_fence_after();
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 1);
                     const uint32_t addr = tmem + lane_addr + 128u * buf;
                     // whole S row into registers first (the four loads overlap), then exponentials and in-place stores
                     uint32_t sv[4][32];
-                    if (!FD_DBG(2)) {
 #pragma unroll
                     for (int qd = 0; qd < 4; ++qd) tmem_ld32(addr + 32 * qd, sv[qd]);
                     tmem_wait_ld();
-                    }
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 2);
-                    if (!FD_DBG(1))
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch) {
                         uint32_t hi[8], lo[8];
@@ -572,17 +379,13 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         for (int i = 0; i < 8; ++i) {
                             const float p0 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i]));
                             const float p1 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i + 1]));
-                            if (MODE == kModeBlock) {
-                                const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
-                                const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
-                                hi[i] = pack_f16x2(h0, h1);
-                                lo[i] = pack_f16x2(p0 - h0, p1 - h1);
-                            } else {
-                                hi[i] = pack_f16x2(p0, p1);
-                            }
+                            const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
+                            const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
+                            hi[i] = pack_f16x2(h0, h1);
+                            lo[i] = pack_f16x2(p0 - h0, p1 - h1);
                         }
                         tmem_st8(addr + 16 * ch, hi);
-                        if (MODE == kModeBlock) tmem_st8(addr + 16 * ch + 8, lo);
+                        tmem_st8(addr + 16 * ch + 8, lo);
                         if (ch == 3) {
                             tmem_wait_st();
                             tc_fence_before();
@@ -590,20 +393,19 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                             if (lane == 0) mbar_arrive(&bars->p_half[buf][t]);
                         }
                     }
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 3);
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->s_done[buf][t]);
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 4);
                     // flush of the accumulator group that ended with the PREVIOUS tile of this row tile (its product
                     // MMA has had a whole tile of time to finish); the last group of the work item is flushed at once
                     if (pending) { ok = do_flush(flush); pending = false; if (!ok) break; }
-                    if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
-                        if (j + 1 == num_jt) { ok = do_flush(j % flush + 1); if (!ok) break; }
+                    ++in_group;
+                    if (in_group == flush || j + 1 == num_jt) {
+                        if (j + 1 == num_jt) { ok = do_flush(in_group); if (!ok) break; }
                         else pending = true;
+                        in_group = 0;
                     }
-                    if (w == 0 && wq == 0 && lane == 0) FD_TRACE(1 + t, j, 5);
                 }
                 if (ok && row < p.Nrow) {
                     const float l = p.left ? p.left[row] : 1.0f;
@@ -617,313 +419,6 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 }
             }
             gn0 += (uint32_t)tiles_per_item;
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 8) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
-    }
-}
-
-// ------------------------------------------------------------------------------------------------ block-mode kernel
-// One 128-row tile per CTA.  Both warpgroups work on the SAME S tile (warpgroup h takes its columns [64 h, 64 h + 64)),
-// so all three ring buffers (3 x 128 TMEM columns) serve this one row tile and the remaining 128 columns hold a
-// double-width accumulator.  That allows the product of a K step to be issued as
-//     [Y_hh | Y_hl] += P_hi [W_hi | W_lo]      (one MMA, N = 2 BT: W_hi and W_lo tiles are adjacent in shared memory)
-//      Y_hh         += P_lo  W_hi              (one MMA, N = BT)
-// i.e. two MMAs instead of three and a wide one instead of two narrow ones (an M128 N64 K16 MMA takes ~50 clk, an
-// N128 one 64 clk).  The flush adds Y_hh + Y_hl into registers.  One product issuer, one Gram issuer.
-template <int BT, int FAST>
-struct SmemB {
-    static constexpr int kXChunk = 128 * 64;
-    static constexpr int kWHalf = BT * 128;                          // 64 j x BT columns fp16
-    static constexpr int kWBytes = (FAST ? 2 : 4) * kWHalf;           // block: [hi h0][lo h0][hi h1][lo h1]; fast: [hi h0][hi h1]
-    static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
-    static __host__ __device__ constexpr int total(int K16) {
-        return 1024 + kStages * stage_bytes(K16) + K16 * kXChunk + 1024;
-    }
-};
-
-struct BarriersB {
-    uint64_t full[kStages], empty[kStages];
-    uint64_t xfull, xempty;
-    uint64_t s_full[3];                     // S tile ready (Gram issuer -> both warpgroups)
-    uint64_t p_done[3][2];                  // warpgroup h has written its half of P in place
-    uint64_t kw_done[3];                    // product MMAs that read this buffer have completed
-    uint64_t y_full, y_empty;               // accumulator flush hand-off
-    uint32_t tmem_base;
-    int abort_flag;
-};
-
-template <int BT, int FAST>
-__global__ void __launch_bounds__(384, 1)
-k_tcb(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUtensorMap map_xcol,
-      const __grid_constant__ CUtensorMap map_whi, const __grid_constant__ CUtensorMap map_wlo, const TcParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    using SM = SmemB<BT, FAST>;
-    constexpr int NBUF = 3;
-    constexpr uint32_t kYCol = 384;                    // accumulator: columns [384, 384 + 2 BT): Y_hh then Y_hl
-    const int K16 = p.K16;
-    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* stage_base = base;
-    uint8_t* xi_base = base + kStages * SM::stage_bytes(K16);
-    BarriersB* bars = (BarriersB*)(xi_base + K16 * SM::kXChunk);
-    volatile int* abort_flag = &bars->abort_flag;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
-        for (int u = 0; u < 3; ++u) {
-            mbar_init(&bars->s_full[u], 1); mbar_init(&bars->kw_done[u], 1);
-            mbar_init(&bars->p_done[u][0], 4); mbar_init(&bars->p_done[u][1], 4);
-        }
-        mbar_init(&bars->y_full, 1); mbar_init(&bars->y_empty, 8);
-        bars->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 8) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = bars->tmem_base;
-
-    // work items: (column chunk c, row tile r), c outermost, r = blockIdx.x + k * gridDim.x (see k_tc)
-    const int my_rows = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_items = my_rows * p.num_chunks;
-    const int flush = p.flush;
-#define FD_ITEM_B(w)                                                                                \
-    const int cch = (w) / my_rows;                                                                  \
-    const int item = (int)blockIdx.x + ((w) % my_rows) * (int)gridDim.x;                            \
-    const int j0 = cch * p.jt_chunk;                                                                \
-    const int num_jt = (p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk;                   \
-    (void)item; (void)cch; (void)j0
-
-    if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(40));
-      if (warp == 8) {
-        // =============================================================== TMA producer
-        if (lane == 0) {
-            prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol); prefetch_tmap(&map_whi);
-            if (!FAST) prefetch_tmap(&map_wlo);
-            uint32_t it = 0;
-            bool ok = true;
-            for (int w = 0; w < my_items && ok; ++w) {
-                FD_ITEM_B(w);
-                ok = mbar_wait(&bars->xempty, (w & 1) ^ 1, abort_flag, p.status, 1);
-                if (!ok) break;
-                mbar_expect_tx(&bars->xfull, K16 * SM::kXChunk);
-                for (int c = 0; c < K16; ++c)
-                    tma_load_2d(xi_base + c * SM::kXChunk, &map_xrow, 0, (int)(c * p.np_rows + (int64_t)item * 128), &bars->xfull);
-                for (int j = 0; j < num_jt; ++j, ++it) {
-                    const int s = it % kStages;
-                    ok = mbar_wait(&bars->empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.status, 2);
-                    if (!ok) break;
-                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
-                    mbar_expect_tx(&bars->full[s], SM::stage_bytes(K16));
-                    for (int c = 0; c < K16; ++c)
-                        tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)(j0 + j) * 128), &bars->full[s]);
-                    uint8_t* wst = st + K16 * SM::kXChunk;
-                    const int x0 = (j0 + j) * 128;
-                    if (FAST) {
-                        tma_load_2d(wst, &map_whi, x0, 0, &bars->full[s]);
-                        tma_load_2d(wst + SM::kWHalf, &map_whi, x0 + 64, 0, &bars->full[s]);
-                    } else {
-                        tma_load_2d(wst, &map_whi, x0, 0, &bars->full[s]);
-                        tma_load_2d(wst + SM::kWHalf, &map_wlo, x0, 0, &bars->full[s]);
-                        tma_load_2d(wst + 2 * SM::kWHalf, &map_whi, x0 + 64, 0, &bars->full[s]);
-                        tma_load_2d(wst + 3 * SM::kWHalf, &map_wlo, x0 + 64, 0, &bars->full[s]);
-                    }
-                }
-            }
-            if (!ok) {
-                const uint32_t issued = it;
-                for (uint32_t k = (issued > (uint32_t)kStages ? issued - kStages : 0); k < issued; ++k) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(&bars->full[k % kStages], (k / kStages) & 1) && clock64() - t0 < 20000000ll) {}
-                }
-            }
-        }
-      } else if (warp == 10) {
-        // =============================================================== Gram MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_g = idesc_f16(128);
-            uint32_t it = 0, g = 0;
-            bool ok = true;
-            for (int w = 0; w < my_items && ok; ++w) {
-                FD_ITEM_B(w);
-                ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
-                if (!ok) break;
-                for (int j = 0; j < num_jt && ok; ++j, ++it, ++g) {
-                    const int s = it % kStages, buf = g % NBUF;
-                    ok = mbar_wait(&bars->kw_done[buf], ((g / NBUF) & 1) ^ 1, abort_flag, p.status, 5);
-                    if (!ok) break;
-                    ok = mbar_wait(&bars->full[s], (it / kStages) & 1, abort_flag, p.status, 4);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t s_addr = tmem + 128u * buf;
-                    uint8_t* st = stage_base + s * SM::stage_bytes(K16);
-                    // small cross terms first, the large hi x hi term last (each MMA rounds at its largest addend)
-                    for (int c = 0; c < K16; ++c) {
-                        const uint64_t a = smem_desc(smem_u32(xi_base + c * SM::kXChunk), 512, 4);
-                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
-                        mma_ss(s_addr, a, b + 2, idesc_g, c > 0);
-                        mma_ss(s_addr, a + 2, b, idesc_g, 1);
-                    }
-                    for (int c = 0; c < K16; ++c) {
-                        const uint64_t a = smem_desc(smem_u32(xi_base + c * SM::kXChunk), 512, 4);
-                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
-                        mma_ss(s_addr, a, b, idesc_g, 1);
-                    }
-                    tc_commit(&bars->s_full[buf]);
-                }
-                if (ok) tc_commit(&bars->xempty);
-            }
-        }
-      } else if (warp == 9) {
-        // =============================================================== product MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_cat = idesc_f16(FAST ? BT : 2 * BT);
-            constexpr uint32_t idesc_y = idesc_f16(BT);
-            uint32_t it = 0, g = 0, n_grp = 0;
-            bool ok = true;
-            const uint32_t y_addr = tmem + kYCol;
-            for (int w = 0; w < my_items && ok; ++w) {
-                FD_ITEM_B(w);
-                for (int j = 0; j < num_jt && ok; ++j, ++it, ++g) {
-                    const int s = it % kStages, buf = g % NBUF;
-                    const uint32_t ph = (g / NBUF) & 1;
-                    const bool group_start = (j % flush) == 0;
-                    const bool group_end = ((j + 1) % flush) == 0 || j + 1 == num_jt;
-                    const uint32_t wst = smem_u32(stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk);
-                    const uint32_t p_addr = tmem + 128u * buf;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        ok = mbar_wait(&bars->p_done[buf][h], ph, abort_flag, p.status, 7);
-                        if (!ok) break;
-                        if (h == 0 && group_start && n_grp > 0) {
-                            ok = mbar_wait(&bars->y_empty, (n_grp - 1) & 1, abort_flag, p.status, 6);
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
-                        // W tiles of column half h: [W_hi | W_lo] adjacent (block) or W_hi alone (fast)
-                        const uint64_t bd = smem_desc(wst + (FAST ? 1 : 2) * h * SM::kWHalf, 1024, 2);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const int ks = 4 * h + k;
-                            mma_ts(y_addr, p_addr + 16 * ks, bd + 2 * k, idesc_cat, !(group_start && ks == 0));
-                            if (!FAST) mma_ts(y_addr, p_addr + 16 * ks + 8, bd + 2 * k, idesc_y, 1);
-                        }
-                    }
-                    if (!ok) break;
-                    tc_commit(&bars->kw_done[buf]);
-                    if (group_end) { tc_commit(&bars->y_full); ++n_grp; }
-                    tc_commit(&bars->empty[s]);
-                }
-            }
-        }
-      }
-    } else {
-        // =============================================================== exponential warpgroups
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(232));
-        const int h = warp >> 2;                       // column half of every tile this warpgroup takes
-        const int wq = warp & 3;
-        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-        const int row_in_tile = wq * 32 + lane;
-        constexpr int YC = BT / 2;                     // accumulator columns per thread: [YC h, YC h + YC)
-        uint32_t g = 0, n_grp = 0;
-        bool ok = true;
-        for (int w = 0; w < my_items && ok; ++w) {
-            FD_ITEM_B(w);
-            const int64_t row = (int64_t)item * 128 + row_in_tile;
-            float acc[YC];
-#pragma unroll
-            for (int c = 0; c < YC; ++c) acc[c] = 0.f;
-            bool pending = false;
-            // Flush: adds the TMEM accumulator into registers and hands it back.  The tensor core accumulates with
-            // round-toward-zero; n same-sign additions lose n / 4 ulp on average (measured 2.85e-8 each vs 2^-25), which the
-            // flush adds back: Y_hh receives two additions per K step (one in fast mode), Y_hl one.
-            auto do_flush = [&](int tiles_in_group) -> bool {
-                const float c_hh = 1.0f + (float)(tiles_in_group * 8 * (FAST ? 1 : 2)) * 2.98023224e-8f;
-                const float c_hl = 1.0f + (float)(tiles_in_group * 8) * 2.98023224e-8f;
-                if (!mbar_wait(&bars->y_full, n_grp & 1, abort_flag, p.status, 10)) return false;
-                ++n_grp;
-                tc_fence_after();
-                const uint32_t yaddr = tmem + lane_addr + kYCol + YC * h;
-                constexpr int NL = YC >= 16 ? YC / 16 : 1;
-                uint32_t vh[NL][16], vl[NL][16];
-#pragma unroll
-                for (int c0 = 0; c0 < NL; ++c0) tmem_ld16(yaddr + 16 * c0, vh[c0]);
-                if (!FAST) {
-#pragma unroll
-                    for (int c0 = 0; c0 < NL; ++c0) tmem_ld16(yaddr + BT + 16 * c0, vl[c0]);
-                }
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->y_empty);
-#pragma unroll
-                for (int c = 0; c < YC; ++c) {
-                    acc[c] = fmaf(__uint_as_float(vh[c / 16][c % 16]), c_hh, acc[c]);
-                    if (!FAST) acc[c] = fmaf(__uint_as_float(vl[c / 16][c % 16]), c_hl, acc[c]);
-                }
-                return true;
-            };
-            for (int j = 0; j < num_jt && ok; ++j, ++g) {
-                const int buf = g % NBUF;
-                ok = mbar_wait(&bars->s_full[buf], (g / NBUF) & 1, abort_flag, p.status, 9);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t addr = tmem + lane_addr + 128u * buf + 64u * h;
-                uint32_t sv[2][32];
-                tmem_ld32(addr, sv[0]);
-                tmem_ld32(addr + 32, sv[1]);
-                tmem_wait_ld();
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t hi[8], lo[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float p0 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i]));
-                        const float p1 = ex2f(__uint_as_float(sv[ch >> 1][16 * (ch & 1) + 2 * i + 1]));
-                        if (!FAST) {
-                            const float h0 = __uint_as_float(__float_as_uint(p0) & 0xFFFFE000u);
-                            const float h1 = __uint_as_float(__float_as_uint(p1) & 0xFFFFE000u);
-                            hi[i] = pack_f16x2(h0, h1);
-                            lo[i] = pack_f16x2(p0 - h0, p1 - h1);
-                        } else {
-                            hi[i] = pack_f16x2(p0, p1);
-                        }
-                    }
-                    tmem_st8(addr + 16 * ch, hi);
-                    if (!FAST) tmem_st8(addr + 16 * ch + 8, lo);
-                }
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->p_done[buf][h]);
-                if (pending) { ok = do_flush(flush); pending = false; if (!ok) break; }
-                if (((j + 1) % flush) == 0 || j + 1 == num_jt) {
-                    if (j + 1 == num_jt) { ok = do_flush(j % flush + 1); if (!ok) break; }
-                    else pending = true;
-                }
-            }
-            if (ok && row < p.Nrow) {
-                const float l = p.left ? p.left[row] : 1.0f;
-#pragma unroll
-                for (int c = 0; c < YC; ++c) {
-                    const int col = YC * h + c;
-                    if (col < p.b) {
-                        float* o = p.Y + row + (int64_t)col * p.ldy;
-                        const float v = acc[c] * l * p.colscale_inv[col];
-                        *o = cch == 0 ? v : *o + v;
-                    }
-                }
-            }
         }
     }
     tc_fence_before();
@@ -1097,17 +592,6 @@ fd_status launch_tc(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, con
     return FD_OK;
 }
 
-template <int BT, int FAST>
-fd_status launch_tcb(fd_ctx* c, const CUtensorMap& mr, const CUtensorMap& mc, const CUtensorMap& mh, const CUtensorMap& ml,
-                     const TcParams& p, int grid) {
-    const int smem = SmemB<BT, FAST>::total(p.K16);
-    if (smem > 227 * 1024) return fail(c, FD_ERR_UNSUPPORTED, "tensor-core kernel needs %d B of shared memory", smem);
-    FD_CUDA(c, cudaFuncSetAttribute(k_tcb<BT, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    k_tcb<BT, FAST><<<grid, 384, smem, c->stream>>>(mr, mc, mh, ml, p);
-    FD_LAUNCH_CHECK(c, "k_tcb");
-    return FD_OK;
-}
-
 }  // namespace
 
 bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
@@ -1164,8 +648,6 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.num_chunks = (int)ceil_div(p.num_jt, p.jt_chunk);
     p.np_rows = NP; p.np_cols = NP; p.K16 = K16;
     p.left = a.left; p.status = status;
-    p.dbg = c->opt_trace >> 1;
-    p.trace = (c->opt_trace & 1) ? reinterpret_cast<long long*>(c->at<char>(L.part)) : nullptr;   // tuning aid: stamps land in the split-partials scratch
     p.flush = c->opt_flush > 0 ? c->opt_flush : 1;
     const int grid = std::min(p.num_work, c->sm_count);
 
@@ -1195,20 +677,18 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
                 !make_map_2d(&ml, wt_lo, (uint64_t)NP, (uint64_t)BT, (uint64_t)NP * 2, 64, BT, CU_TENSOR_MAP_SWIZZLE_128B))
                 return fail(c, FD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the block operands");
             p.b = bc; p.colscale_inv = inv; p.Y = a.Y + (int64_t)c0 * a.ldy; p.ldy = a.ldy;
-            TcParams pb = p;                       // one-row-tile variant: 128-row work items
-            pb.num_work = (int)ceil_div(a.Nrow, 128);
-            const int grid_b = std::min(pb.num_work, c->sm_count);
-            const bool one_tile = c->opt_tc_variant != 1;
-#define FD_TC_CASE(B)                                                                              \
-    case B:                                                                                        \
-        if (one_tile) {                                                                            \
-            if (fast) FD_TRY((launch_tcb<B, 1>(c, mr, mc, mh, ml, pb, grid_b)));                   \
-            else FD_TRY((launch_tcb<B, 0>(c, mr, mc, mh, ml, pb, grid_b)));                        \
-        } else if (fast) FD_TRY((launch_tc<B, kModeFast>(c, mr, mc, mh, ml, p, grid)));            \
-        else FD_TRY((launch_tc<B, kModeBlock>(c, mr, mc, mh, ml, p, grid)));                       \
-        break;
-            switch (BT) { FD_TC_CASE(16) FD_TC_CASE(32) FD_TC_CASE(64) }
-#undef FD_TC_CASE
+            if (fast) {
+                // reduced-precision mode (single fp16 operands): the one-row-tile kernel with sixteen exponential warps
+                TcParams pb = p;                   // 128-row work items
+                pb.num_work = (int)ceil_div(a.Nrow, 128);
+                FD_TRY(launch_fast_product(c, BT, mr, mc, mh, pb, std::min(pb.num_work, c->sm_count)));
+                continue;
+            }
+            switch (BT) {
+                case 16: FD_TRY((launch_tc<16, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+                case 32: FD_TRY((launch_tc<32, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+                default: FD_TRY((launch_tc<64, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+            }
         }
     }
     return FD_OK;

@@ -88,6 +88,44 @@ def test_fast_mode(fd, dev):
     assert err > 1e-6            # it really is the reduced-precision path
 
 
+# The reduced-precision mode has a kernel of its own (one row tile per CTA, three exponent buffers, tiles alternating
+# between two pairs of warpgroups): the same edge shapes as the fp32-grade kernel, against the oracle at its 3e-3 bound.
+@pytest.mark.parametrize("N", [1, 100, 128, 129, 257, 1000, 2304])
+def test_fast_mode_row_and_column_tails(fd, dev, N):
+    tc_case(fd, dev, workloads.torus6(N, seed=N), 2.0, 1.0, 64 if N > 1 else 1, prec=1)
+
+
+@pytest.mark.parametrize("b", [1, 8, 16, 24, 32, 40, 64, 70, 128])
+def test_fast_mode_block_widths(fd, dev, b):
+    tc_case(fd, dev, workloads.torus6(900, seed=b), 1.0, 1.0, b, prec=1)
+
+
+@pytest.mark.parametrize("D,beta", [(2, 3.0), (12, 2.0), (20, 1.0), (30, 1.0)])
+def test_fast_mode_dimensions_and_k_slabs(fd, dev, D, beta):
+    X = workloads.latent_torus(1200, seed=D, D=D) if D >= 13 else workloads.gaussian_cloud(1200, D, seed=D, scale=0.7)
+    tc_case(fd, dev, X, beta, 1.0, 32, prec=1)
+
+
+@pytest.mark.parametrize("opts", [{"flush": 1}, {"flush": 3}, {"flush": 64}, {"jt_chunk": 1}, {"jt_chunk": 2}, {"jt_chunk": 5, "flush": 2}])
+def test_fast_mode_flush_groups_and_column_chunks(fd, dev, opts):
+    # 3000 points = 24 column tiles: group and chunk tails, odd tile counts per chunk (the running tile index carries the
+    # buffer and warpgroup rotation across work items), and run-to-run bit-reproducibility
+    X = workloads.torus6(3000, seed=9)
+    V = workloads.block(3000, 64, seed=2)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=64)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    for k, v in opts.items():
+        ctx.set_option(k, v)
+    ctx.degree(2.0, 1.0)
+    Vd = fd.to_colmajor(V, dev)
+    Y1 = ctx.apply(Vd, prec=fd.FD_PREC_FAST).clone()
+    Y2 = ctx.apply(Vd, prec=fd.FD_PREC_FAST)
+    ctx.synchronize()
+    assert torch.equal(Y1, Y2)
+    assert relF(Y1.cpu().numpy(), dense.apply(X, 2.0, 1.0, V)) <= TOL_FAST
+    ctx.close()
+
+
 def test_c4_shape_reduced(fd, dev):
     tc_case(fd, dev, workloads.latent_torus(3000), 2.0, 1.0, 32)
 
