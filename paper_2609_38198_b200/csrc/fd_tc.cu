@@ -172,6 +172,9 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         // =============================================================== Gram MMA issuer (one thread)
         // Issues S(n) = A_t B_j^T for every tile as soon as its ring buffer is free again; runs up to NBUF tiles ahead.
         if (lane == 0) {
+          if constexpr (MODE == kModeRowsum) {
+            // Row-sum mode: the MUFU binds and the tensor pipe is mostly idle; descriptors are rebuilt per MMA, which paces
+            // the Gram MMAs between the warpgroups' TMEM loads (issuing them in tight bursts measured 5 % slower).
             constexpr uint32_t idesc_g = idesc_f16(128);
             uint32_t it0 = 0, gn0 = 0;
             bool ok = true;
@@ -220,6 +223,68 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 it0 += (uint32_t)num_jt;
                 gn0 += (uint32_t)tiles_per_item;
             }
+          } else {
+            constexpr uint32_t idesc_g = idesc_f16(128);
+            // Operand descriptors as (low, high) words and ring positions as counters: this thread shares its scheduler
+            // with busy warps, so every instruction it does not issue shortens the gap between two MMAs.
+            const uint64_t xd = smem_desc(smem_u32(xi_base), 512, 4);      // 64 B rows (SWIZZLE_64B), 512 B between 8-row groups
+            const uint32_t xi_lo = (uint32_t)xd, xdesc_hi = (uint32_t)(xd >> 32);
+            const uint32_t stage_lo = (uint32_t)smem_desc(smem_u32(stage_base), 512, 4);
+            const uint32_t stage_step = (uint32_t)(SM::stage_bytes(K16) >> 4);
+            constexpr uint32_t kSlab = SM::kXChunk >> 4;
+            uint32_t itj = 0, buf = 0, gr = 0, ph = 0;              // column-tile counter; tile index mod NBUF, mod kRingPeriod, ring phase
+            bool first_round = true;                                // no buffer has been used yet
+            bool ok = true;
+            for (int w = 0; w < my_items && ok; ++w) {
+                FD_ITEM_GEOMETRY(w);
+                ok = mbar_wait(&bars->xfull, w & 1, abort_flag, p.status, 3);
+                if (!ok) break;
+                tc_fence_after();
+                for (int n = 0; n < tiles_per_item && ok; ++n) {
+                    const int t = n & 1;
+                    const int s = itj % kStages;
+                    if (!first_round) {
+                        // the tile that used this buffer last (NBUF tiles ago, possibly of the other row tile) must be finished
+                        const int tp = (NBUF & 1) ? (t ^ 1) : t;
+                        const uint32_t php = gr >= (uint32_t)NBUF ? ph : ph ^ 1u;
+                        uint64_t* fb = (MODE == kModeRowsum) ? &bars->s_done[buf][tp] : &bars->kw_done[buf][tp];
+                        ok = mbar_wait(fb, php, abort_flag, p.status, 5);
+                        if (!ok) break;
+                    }
+                    if (t == 0) {
+                        ok = mbar_wait(&bars->full[s], (itj / kStages) & 1, abort_flag, p.status, 4);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    // The two small cross terms (hi x lo) go first and the large hi x hi term last: each MMA rounds its
+                    // result at the magnitude of its largest addend, so only the final one rounds at full magnitude.
+                    const uint32_t s_addr = tmem + 128u * buf;
+                    const uint32_t a0 = xi_lo + (uint32_t)(t * K16) * kSlab, b0 = stage_lo + (uint32_t)s * stage_step;
+                    if (K16 == 1) {
+                        mma_ss2<0>(s_addr, a0, xdesc_hi, b0 + 2, xdesc_hi, idesc_g);          // + 2: the lo half starts 32 B into the row
+                        mma_ss2<1>(s_addr, a0 + 2, xdesc_hi, b0, xdesc_hi, idesc_g);
+                        mma_ss2<1>(s_addr, a0, xdesc_hi, b0, xdesc_hi, idesc_g);
+                    } else {
+                        for (int c = 0; c < K16; ++c) {
+                            const uint32_t a = a0 + (uint32_t)c * kSlab, b = b0 + (uint32_t)c * kSlab;
+                            if (c == 0) mma_ss2<0>(s_addr, a, xdesc_hi, b + 2, xdesc_hi, idesc_g);
+                            else mma_ss2<1>(s_addr, a, xdesc_hi, b + 2, xdesc_hi, idesc_g);
+                            mma_ss2<1>(s_addr, a + 2, xdesc_hi, b, xdesc_hi, idesc_g);
+                        }
+                        for (int c = 0; c < K16; ++c)
+                            mma_ss2<1>(s_addr, a0 + (uint32_t)c * kSlab, xdesc_hi, b0 + (uint32_t)c * kSlab, xdesc_hi, idesc_g);
+                    }
+                    tc_commit(&bars->s_full[buf][t]);
+                    if (t == 1) {
+                        if (MODE == kModeRowsum) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
+                        ++itj;
+                    }
+                    if (++buf == (uint32_t)NBUF) { buf = 0; first_round = false; }
+                    if (++gr == kRingPeriod) { gr = 0; ph ^= 1u; }
+                }
+                if (ok) tc_commit(&bars->xempty);                  // the row operand tiles may be replaced
+            }
+          }
         }
       } else if (MODE != kModeRowsum) {
         // =============================================================== product MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1
@@ -227,17 +292,21 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         if (lane == 0) {
             constexpr uint32_t idesc_y = idesc_f16(BT);
             const int t = warp - 9;
-            uint32_t it0 = 0, gn0 = 0, n_grp = 0;
+            // W stage descriptor as (low, high) words: 128 B rows (SWIZZLE_128B), 1024 B between 8-row groups
+            const uint64_t wd = smem_desc(smem_u32(stage_base + K16 * SM::kXChunk), 1024, 2);
+            const uint32_t wbase_lo = (uint32_t)wd, wdesc_hi = (uint32_t)(wd >> 32);
+            const uint32_t stage_step = (uint32_t)(SM::stage_bytes(K16) >> 4);
+            constexpr uint32_t kLoOff = (uint32_t)((2 * SM::kWHalf) >> 4);          // W_lo tiles follow the two W_hi tiles of a stage
+            uint32_t itj = 0, n_grp = 0;
+            uint32_t buf = (uint32_t)t % NBUF, gr = (uint32_t)t, ph = 0;            // this row tile's tile index mod NBUF, mod kRingPeriod, ring phase
             bool ok = true;
             const uint32_t y_addr = tmem + kYCol + 64 * t;
             for (int w = 0; w < my_items && ok; ++w) {
                 FD_ITEM_GEOMETRY(w);
                 int in_group = 0;                                  // tiles accumulated in the current group (no division in the hot loop)
-                for (int j = 0; j < num_jt && ok; ++j) {
-                    const uint32_t g = gn0 + 2u * (uint32_t)j + (uint32_t)t;
-                    const int buf = g % NBUF;
-                    const int s = (it0 + (uint32_t)j) % kStages;
-                    ok = mbar_wait(&bars->p_half[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 7);
+                for (int j = 0; j < num_jt && ok; ++j, ++itj) {
+                    const int s = itj % kStages;
+                    ok = mbar_wait(&bars->p_half[buf][t], ph, abort_flag, p.status, 7);
                     if (!ok) break;
                     const bool group_start = in_group == 0;
                     const bool group_end = in_group + 1 == flush || j + 1 == num_jt;
@@ -250,30 +319,29 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     // Y_t += P W : 8 K steps of 16 columns j; K step ks reads P_hi at S-buffer columns [16 ks, 16 ks + 8)
                     // and P_lo at [16 ks + 8, 16 ks + 16) (the warpgroup wrote them in place over S).  The first four K steps
                     // start as soon as the first half of P is written, the rest once the tile is complete.
-                    const uint32_t wst = smem_u32(stage_base + s * SM::stage_bytes(K16) + K16 * SM::kXChunk);
-                    const uint64_t bd_hi = smem_desc(wst, 1024, 2);
-                    const uint64_t bd_lo = smem_desc(wst + 2 * SM::kWHalf, 1024, 2);
+                    const uint32_t w_lo = wbase_lo + (uint32_t)s * stage_step;
                     const uint32_t p_addr = tmem + 128u * buf;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         if (ks == 4) {
-                            ok = mbar_wait(&bars->s_done[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 7);
+                            ok = mbar_wait(&bars->s_done[buf][t], ph, abort_flag, p.status, 7);
                             if (!ok) break;
                             tc_fence_after();
                         }
                         const uint32_t off = (uint32_t)(((ks >> 2) * SM::kWHalf + (ks & 3) * 32) >> 4);
                         const uint32_t a_hi = p_addr + 16 * ks;
-                        mma_ts(y_addr, a_hi, bd_hi + off, idesc_y, !(group_start && ks == 0));
-                        mma_ts(y_addr, a_hi + 8, bd_hi + off, idesc_y, 1);
-                        mma_ts(y_addr, a_hi, bd_lo + off, idesc_y, 1);
+                        if (ks == 0 && group_start) mma_ts2<0>(y_addr, a_hi, w_lo + off, wdesc_hi, idesc_y);
+                        else mma_ts2<1>(y_addr, a_hi, w_lo + off, wdesc_hi, idesc_y);
+                        mma_ts2<1>(y_addr, a_hi + 8, w_lo + off, wdesc_hi, idesc_y);
+                        mma_ts2<1>(y_addr, a_hi, w_lo + kLoOff + off, wdesc_hi, idesc_y);
                     }
                     if (!ok) break;
                     tc_commit(&bars->kw_done[buf][t]);
                     if (group_end) { tc_commit(&bars->y_full[t]); ++n_grp; }
                     tc_commit(&bars->empty[s]);
+                    buf += 2; if (buf >= (uint32_t)NBUF) buf -= NBUF;
+                    gr += 2; if (gr >= kRingPeriod) { gr -= kRingPeriod; ph ^= 1u; }
                 }
-                it0 += (uint32_t)num_jt;
-                gn0 += (uint32_t)tiles_per_item;
             }
         }
       }
