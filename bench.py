@@ -1,22 +1,25 @@
 #!/usr/bin/env python
 """Benchmark of the FlashDiffusion hot path on B200.
 
-One step = one pass of the whole hot path at a fixed bandwidth over the headline workload
-(6-torus in R^12, N = 2^20, block b = 64, alpha = 1, beta = 2): degree pass q = K 1, second
-normalisation pass d = q^-a * K q^-a, scale vector s, and the block product Y = M V.  A step
-therefore processes (b + 2) N^2 pair-columns; `value` is that count over the step time,
-aggregated over ranks (each rank runs an independent replica: the path is not sharded).
+Headline metric: kernel-apply throughput N^2 * b / t_apply (pair-columns per second) of the fp32-grade block product
+Y = diag(s) K diag(s) V on the headline workload (6-torus in R^12, N = 2^20, block b = 64, alpha = 1, beta = 2), with
+its fraction of the binding roofline (one exponential per pair on the MUFU).  One timed step is one pass of the whole
+hot path at a fresh bandwidth -- degree pass q = K 1, second normalisation pass d = q^-a * K q^-a, scale vector s, block
+product -- so the step time, the degree passes and the reduced-precision product are reported beside the headline, as
+are the end-to-end figure through the C ABI with host buffers, the CPU float64 oracle on the box's own cores, and the
+time to k eigenpairs on the five benchmark configurations.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--n LOG2N]
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU float64 oracle on a bounded
-row sample of the same workload instead.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU float64 oracle on a bounded row sample of the same
+workload instead.  `--gpus N` without a launcher starts N ranks itself (one per GPU, independent replicas).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -28,16 +31,12 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-METRIC = "kernel-apply pair-columns per second (degree passes + block product, one step)"
+METRIC = "kernel-apply pair-columns per second of the block product Y = M V (N^2 * b / t_apply)"
 UNIT = "pair*cols/s"
 
-# Nominal unit counts for the roofline: MUFU 16 ex2/clk/SM, FMA pipe 128 FFMA/clk/SM, 148 SMs.
-SM_COUNT = 148
-MUFU_PER_CLK_SM = 16
-FMA_PER_CLK_SM = 128
-
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or None.
-NCU_TRAFFIC_BYTES = {"simt": None, "tc": 20.15e9 + 2.18e9}   # k_tc block mode at N = 2^20, profiles/bench_c5_n2e20_launch_list.md
+# DRAM bytes per launch of the timed block-product kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture at N = 2^20, summarised under profiles/), keyed by the kernel that bench times; None = not captured.
+NCU_TRAFFIC_BYTES = {"k_tc<64, block>": None, "k_simt": None}
 
 
 def measured_peaks():
@@ -108,21 +107,28 @@ def workload(log2n: int):
     N = 1 << log2n
     X = workloads.torus6(N, seed=42)
     V = workloads.block(N, 64, seed=1)
-    return X, V, dict(workload=f"C5: 6-torus R^12 + noise 0.01, N=2^{log2n}, b=64, alpha=1, beta=2.0",
+    return X, V, dict(workload=f"C5: 6-torus R^12 + noise 0.01, N=2^{log2n}, b=64, alpha=1, beta=2.0, fp32-grade mode",
                       N=N, D=12, b=64, alpha=1.0, beta=2.0, l2_note="inputs (X, V, Y: >= 0.6 GB) exceed the 126 MB L2")
 
 
 # ------------------------------------------------------------------------------------------- CPU oracle arm
-def oracle_step(X64, V64, beta, alpha, rows, q_hint=None):
-    """One bounded sample of the step on the CPU oracle: the three passes on `rows` rows."""
+def oracle_sample(X64, V64, beta, rows, w):
+    """A bounded sample of the step on the CPU oracle: the three passes on `rows` rows; returns (seconds of the two
+    degree passes, seconds of the block product).  The second pass and the product need q, s on all columns: a positive
+    surrogate vector of the right magnitude stands in (the cost per pair is what is timed, not the values)."""
     from oracle import blocked
-    q_rows, _ = blocked.rows_apply_general(X64, beta, None, rows=rows, want_rowsq=True)
-    # the second pass and the product need q, s on all columns: use a positive surrogate vector of the right
-    # magnitude for the columns (the cost per pair is what is being timed, not the values)
-    w = q_hint
+    t0 = time.perf_counter()
+    blocked.rows_apply_general(X64, beta, None, rows=rows, want_rowsq=True)
     blocked.rows_apply_general(X64, beta, None, rows=rows, left=w, right=w)
+    t1 = time.perf_counter()
     blocked.rows_apply_general(X64, beta, V64, rows=rows, left=w, right=w)
-    return q_rows
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def oracle_rows_for(N, cores, seconds):
+    # ~4e7 pair evaluations per core-second for the b = 64 product on these hosts
+    return int(max(16, min(N, seconds * cores * 2.5e7 / N)))
 
 
 def run_reference(args):
@@ -130,31 +136,31 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import blocked
+    import workloads
     X, V, cfg = workload(args.n)
     N, b = cfg["N"], cfg["b"]
     X64 = X.astype(np.float64)
     V64 = np.ascontiguousarray(V.astype(np.float64))
     cores = blocked.threads()
-    # size the sample for ~6-10 s per step on this host: ~4e7 pair-evaluations per core-second over three passes
-    rows_n = int(max(16, min(N, 6.0 * cores * 2.0e7 / N)))
-    import workloads
+    rows_n = oracle_rows_for(N, cores, 5.0)
     rows = workloads.row_sample(N, rows_n, seed=11)
     w = np.full(N, 1e-2)
-    for _ in range(max(1, min(args.warmup, 1))):
-        oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows[: max(16, rows_n // 8)], w)
+    oracle_sample(X64, V64, cfg["beta"], rows[: max(16, rows_n // 8)], w)
+    t_deg = t_app = 0.0
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows, w)
+        a, c = oracle_sample(X64, V64, cfg["beta"], rows, w)
+        t_deg += a; t_app += c
     dt = (time.perf_counter() - t0) / args.steps
-    units = rows_n * N * (b + 2)
-    value = units / dt
-    sample = f"{rows_n} sampled rows x all {N} columns, three passes (b = 1, 1, {b}), float64, rows.c + OpenMP"
+    value = rows_n * float(N) * b / (t_app / args.steps)
+    sample = (f"{rows_n} sampled rows x all {N} columns per step: block product (b = {b}) timed for the metric, the two "
+              f"degree passes beside it; float64, rows.c + OpenMP")
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-           "gpu_launches": 0}
+           "whole_step": {"pair_cols_per_s": rows_n * float(N) * (b + 2) / dt}, "gpu_launches": 0}
     print(json.dumps(out), flush=True)
 
 
@@ -173,12 +179,25 @@ def job_value(units_per_rank: float, world: int, ms: float) -> float:
     return units_per_rank * world / (ms * 1e-3)
 
 
+def free_port() -> int:
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def spawn_ranks(args) -> int:
+    """`python bench.py --gpus N` without a launcher: start N local ranks (one per GPU) of this same script."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 # ------------------------------------------------------------------------------------------- GPU arm
 def run_gpu(args):
     import torch
+    import __graft_entry__ as entry
+    entry.build()
     import paper_2609_38198_b200 as fd
-    from paper_2609_38198_b200 import build as fd_build
-    fd_build.build()
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -243,6 +262,25 @@ def run_gpu(args):
     total_ms = t_start.elapsed_time(t_end)
     deg_ms = float(np.mean([a.elapsed_time(b_) for a, b_, _ in timers]))
     app_ms = float(np.mean([b_.elapsed_time(c_) for _, b_, c_ in timers]))
+    path_used = "tc" if ctx.get_option("last_path") == 2 else "simt"
+
+    # SM clock the block-product kernel actually ran at: SM cycles of its first CTA over the kernel's duration
+    sustained_mhz = None
+    if path_used == "tc":
+        e0, e1 = ev(), ev()
+        e0.record(stream); ctx.apply(Vd, out=Yd); e1.record(stream)
+        torch.cuda.synchronize(dev)
+        sustained_mhz = ctx.get_option("tc_cycles") / (e0.elapsed_time(e1) * 1e3)
+    # the reduced-precision product, reported separately (three repeats)
+    fast_ms = None
+    if path_used == "tc":
+        ts = []
+        for _ in range(3):
+            e0, e1 = ev(), ev()
+            e0.record(stream); ctx.apply(Vd, out=Yd, prec=fd.FD_PREC_FAST); e1.record(stream)
+            torch.cuda.synchronize(dev)
+            ts.append(e0.elapsed_time(e1))
+        fast_ms = float(np.median(ts))
 
     # end-to-end through the public API with host buffers: H2D of X and V, D2H of Y every step
     def e2e_step():
@@ -270,35 +308,51 @@ def run_gpu(args):
 
     total_ms, e2e_ms, deg_ms, app_ms = max_over_ranks([total_ms, e2e_ms, deg_ms, app_ms], dist, dev)
     step_ms = total_ms / args.steps
-    units = float(N) * N * (b + 2)
+    units = float(N) * N * b                      # pair-columns of one block product
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        path_used = "tc" if ctx.get_option("last_path") == 2 else "simt"
-        pairs_per_s = float(N) * N / (app_ms * 1e-3)
-        mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
-        mufu_peak = SM_COUNT * MUFU_PER_CLK_SM * peaks.get("sm_max_mhz", 1965.0) * 1e6       # exp / s
-        fma_peak = SM_COUNT * FMA_PER_CLK_SM * peaks.get("sm_max_mhz", 1965.0) * 1e6         # FMA / s
+        rates = fd.fd_unit_peaks(dev)
         D = cfg["D"]
+        sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+        pairs_per_s = float(N) * N / (app_ms * 1e-3)
+        mufu_peak = rates["sm_count"] * rates["ex2_per_clk_sm"] * sm_max * 1e6         # exp / s at the maximum SM clock
+        fma_peak = rates["sm_count"] * rates["ffma_per_clk_sm"] * sm_max * 1e6
         if path_used == "simt":
             # everything on the FMA pipe: per pair 2 D (difference form) + b (product) + ~3 issue slots
             peak_pairs = fma_peak / (2 * D + b + 3)
             binder = "fma_pipe (direct-difference distance + block product on FFMA)"
+            kernel_name = "k_simt"
         else:
             peak_pairs = mufu_peak
-            binder = "mufu (one ex2 per pair)"
-        roofline = {"bound": "alu", "kernel": "block product Y = M V (dominant kernel)", "binder": binder,
+            binder = "mufu (one ex2 per pair; distance and product on the tensor cores)"
+            kernel_name = "k_tc<64, block>"
+        roofline = {"bound": "alu", "kernel": f"{kernel_name}: block product Y = M V (dominant kernel)", "binder": binder,
                     "achieved": pairs_per_s / 1e9, "peak": peak_pairs / 1e9, "unit": "Gpairs/s",
-                    "frac": pairs_per_s / peak_pairs, "peak_source": f"unit counts x {peak_kind} max SM clock",
-                    "mufu_floor_frac": pairs_per_s / mufu_peak, "traffic": NCU_TRAFFIC_BYTES.get(path_used) if N == (1 << 20) else None,
+                    "frac": pairs_per_s / peak_pairs,
+                    "peak_source": (f"measured unit rate ({rates['ex2_per_clk_sm']:.2f} ex2/clk/SM, {rates['sm_count']} SMs; "
+                                    f"fd_unit_peaks in this run) x maximum SM clock {sm_max:.0f} MHz ({peak_kind})"),
+                    "sustained_sm_mhz": sustained_mhz,
+                    "frac_at_sustained_clock": (pairs_per_s / (peak_pairs * sustained_mhz / sm_max)) if sustained_mhz else None,
+                    "traffic": NCU_TRAFFIC_BYTES.get(kernel_name) if N == (1 << 20) else None,
                     "algorithmic_bytes": 4.0 * N * (D + 2 * b + 2),
-                    "sm_mhz_seen": mhz}
-        out = {"metric": METRIC, "value": job_value(units, world, step_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                    "tensor_work_per_tile_clk": {"gram_3_mma_ss_n128": 3 * rates["clk_mma_ss_n128"],
+                                                 "product_24_mma_ts_n64": 24 * rates["clk_mma_ts_n64"],
+                                                 "mufu_128x128_exps": 128 * 128 / rates["ex2_per_clk_sm"]},
+                    "unit_rates": rates}
+        deg_pairs_per_s = 2.0 * float(N) * N / (deg_ms * 1e-3)
+        out = {"metric": METRIC, "value": job_value(units, world, app_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
-               "apply_only": {"ms": app_ms, "pair_cols_per_s": float(N) * N * b / (app_ms * 1e-3), "pairs_per_s": pairs_per_s},
-               "degree_ms": deg_ms, "path": path_used, "roofline": roofline,
+               "apply_ms": app_ms, "path": path_used, "roofline": roofline,
+               "whole_step": {"ms": step_ms, "pair_cols_per_s": job_value(float(N) * N * (b + 2), world, step_ms),
+                              "note": "degree pass + second normalisation pass + scale vector + block product"},
+               "degree_passes": {"ms_both": deg_ms, "pairs_per_s": deg_pairs_per_s, "frac_of_mufu_peak": deg_pairs_per_s / mufu_peak},
+               "fast_mode_apply": None if fast_ms is None else {
+                   "ms": fast_ms, "pair_cols_per_s": units / (fast_ms * 1e-3), "frac_of_mufu_peak": float(N) * N / (fast_ms * 1e-3) / mufu_peak,
+                   "note": "FD_PREC_FAST: single fp16 operands, relative Frobenius error ~2e-4 (bound 3e-3); reported separately"},
                "e2e": {"value": job_value(units, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+                       "note": "host buffers: H2D of X and V, fd_create, degree passes, block product, D2H of Y",
                        "h2d_bytes_per_step": int(Xh.numel() * 4 + Vh.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 4)},
                "gpu_launches": int(launches), "workspace_bytes": ctx.workspace_bytes}
         if not args.no_cpu:
@@ -307,7 +361,7 @@ def run_gpu(args):
         if not args.no_eigs:
             del Xd, Vd, Yd
             torch.cuda.empty_cache()
-            out["time_to_k_eigs"] = time_to_k_eigs(fd, dev, full=args.eigs_full)
+            out["time_to_k_eigs"] = time_to_k_eigs(fd, dev, args)
         print(json.dumps(out), flush=True)
     ctx.close()
     if dist is not None:
@@ -315,35 +369,38 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-def time_to_k_eigs(fd, dev, full=False):
-    """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs) on the
-    benchmark configurations at full size (C1, C2 at beta = 10 and 30, C3, C4; with --eigs-full also C5 at N = 2^20), the
-    whole dyadic bandwidth flow on C3, and the nested-level ladder.  Host wall clock around synchronous calls."""
+def time_to_k_eigs(fd, dev, args):
+    """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs) on the five
+    benchmark configurations at their full sizes (C2 at all four bandwidths; non-convergence within the apply budget is a
+    reported outcome there), the whole dyadic bandwidth flow on C3, and the nested-level ladder with the bandwidth
+    re-optimised on every level.  Host wall clock around synchronous calls."""
     import torch
     import workloads
     res = []
-    # (name, points, k, b, beta): the five benchmark configurations at their full sizes
-    cases = [("C1 circle", workloads.circle(2048), 8, 8, 200.0),
-             ("C2 2-torus", workloads.torus2(16384, seed=42), 32, 16, 10.0),
-             ("C2 2-torus", None, 32, 16, 30.0),
-             ("C3 6-torus", workloads.torus6(1 << 17, seed=42), 64, 32, 2.0),
-             ("C4 latent torus R^30", workloads.latent_torus(262144, seed=42), 32, 32, 2.0)]
-    if full:
-        cases.append(("C5 6-torus", workloads.torus6(1 << 20, seed=42), 128, 64, 2.0))
+    # (name, points, k, b, beta, max_applies)
+    cases = [("C1 circle", workloads.circle(2048), 8, 8, 200.0, 600),
+             ("C2 2-torus", workloads.torus2(16384, seed=42), 32, 16, 10.0, 600),
+             ("C2 2-torus", None, 32, 16, 30.0, 600),
+             ("C2 2-torus", None, 32, 16, 100.0, 1000),
+             ("C2 2-torus", None, 32, 16, 300.0, 1000),
+             ("C3 6-torus", workloads.torus6(1 << 17, seed=42), 64, 32, 2.0, 600),
+             ("C4 latent torus R^30", workloads.latent_torus(262144, seed=42), 32, 32, 2.0, 600)]
+    if not args.no_c5_eigs:
+        cases.append(("C5 6-torus", workloads.torus6(1 << 20, seed=42), 128, 64, 2.0, 400))
     Xnp = None
-    for name, Xc, k, b, beta in cases:
+    for name, Xc, k, b, beta, max_applies in cases:
         if Xc is not None:
             Xnp = Xc
         N = Xnp.shape[0]
         X = torch.from_numpy(Xnp).to(dev)
-        m_max = (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
+        m_max = default_m_max(k, b)
         ctx = fd.Context(X, b_max=b, m_max=m_max)
         ctx.degree(beta, 1.0)                                        # warm-up of both passes
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
         ctx.degree(beta, 1.0)
         t1 = time.perf_counter()
-        lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=600, allow_not_converged=True)
+        lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=max_applies, allow_not_converged=True)
         t2 = time.perf_counter()
         rec = {"workload": f"{name}: N={N}, D={Xnp.shape[1]}, k={k}, b={b}, alpha=1, beta={beta}, tol=1e-6",
                "path": "tc" if ctx.get_option("last_path") == 2 else "simt", "degree_s": t1 - t0,
@@ -362,46 +419,52 @@ def time_to_k_eigs(fd, dev, full=False):
         del ctx, X
         torch.cuda.empty_cache()
         res.append(rec)
-    res.append(ladder(fd, dev, full))
+    res.append(ladder(fd, dev, args.ladder_full))
     return res
 
 
+def default_m_max(k, b):
+    return (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
+
+
 def ladder(fd, dev, full=False):
-    """The (n, beta) continuation of Sec. 1 at fixed beta = 2: nested levels (first n rows of one draw), each level's solve
-    warm-started from the previous level's eigenpairs through the out-of-sample extension (fd_ladder_start), with the
-    cold-started solve of the same level beside it.  Default: 2^15 -> 2^16 -> 2^17 (k = 64, b = 32); --eigs-full: the
-    2^16 ... 2^20 ladder with k = 128, b = 64."""
+    """The (n, beta) continuation of Sec. 1: nested levels (first n rows of one draw).  On every level the bandwidth is
+    re-optimised by the dyadic flow started one probe below the previous level's beta_x, and every probe's solve is
+    warm-started: the first from the previous level's eigenpairs through the out-of-sample extension (fd_ladder_start),
+    the others from the previous probe.  A cold-started solve at the level's beta_x stands beside it.
+    Default: 2^15 -> 2^16 -> 2^17 (k = 64, b = 32); --ladder-full: config 5 itself, 2^16 ... 2^20 with k = 128, b = 64."""
     import torch
     import workloads
     levels, k, b = ([1 << e for e in range(16, 21)], 128, 64) if full else ([1 << 15, 1 << 16, 1 << 17], 64, 32)
     Xall = torch.from_numpy(workloads.torus6(levels[-1], seed=42)).to(dev)
-    m_max = (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
-    out = {"workload": f"6-torus ladder N = {levels}, k={k}, b={b}, alpha=1, beta=2.0, tol=1e-6", "levels": []}
+    m_max = default_m_max(k, b)
+    out = {"workload": f"6-torus ladder N = {levels}, k={k}, b={b}, alpha=1, tol=1e-6, beta re-optimised per level", "levels": []}
     prev = None
     t_all = time.perf_counter()
     for n in levels:
         X = Xall[:n]
         ctx = fd.Context(X, b_max=b, m_max=m_max)
-        t0 = time.perf_counter()
-        ctx.degree(2.0, 1.0)
         rec = {"N": n}
-        if prev is not None:
-            pctx, plam, pU = prev
-            Q0 = ctx.ladder_start(pctx, X, pU, plam)
-            t1 = time.perf_counter()
-            lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=400, Q0=Q0, allow_not_converged=True)
-            rec.update(extend_s=t1 - t0, warm_s=time.perf_counter() - t1, warm_applies=int(info.applies),
-                       warm_converged=int(info.converged))
-            pctx.close()
-        t2 = time.perf_counter()
-        lam_c, U_c, info_c = ctx.eigs(k, b, tol=1e-6, max_applies=400, allow_not_converged=True)
-        rec.update(cold_s=time.perf_counter() - t2, cold_applies=int(info_c.applies), cold_converged=int(info_c.converged))
+        t0 = time.perf_counter()
         if prev is None:
-            lam, U = lam_c, U_c
+            bx, outcome, lam, U, recs = ctx.beta_flow(k, b, 1.0, beta_start=0.5, beta_max=64.0, tol=1e-6, max_applies=400)
         else:
-            rec["max_eval_diff_warm_vs_cold"] = float(abs(lam - lam_c).max())
+            pctx, plam, pU, pbx = prev
+            ctx.degree(pbx, 1.0)                                    # the extension is scaled by this level's degrees
+            Q0 = ctx.ladder_start(pctx, X, pU, plam)
+            rec["extend_s"] = time.perf_counter() - t0
+            bx, outcome, lam, U, recs = ctx.beta_flow(k, b, 1.0, beta_start=pbx / 2.0, beta_max=pbx * 16.0, tol=1e-6,
+                                                      max_applies=400, Q0=Q0)
+            pctx.close()
+        rec.update(flow_s=time.perf_counter() - t0, beta_x=bx, outcome=outcome, probes=len(recs),
+                   flow_applies=int(sum(r["applies"] for r in recs)), probe_betas=[r["beta"] for r in recs])
+        t2 = time.perf_counter()
+        ctx.degree(bx, 1.0)
+        lam_c, U_c, info_c = ctx.eigs(k, b, tol=1e-6, max_applies=400, allow_not_converged=True)
+        rec.update(cold_at_beta_x_s=time.perf_counter() - t2, cold_applies=int(info_c.applies), cold_converged=int(info_c.converged),
+                   max_eval_diff_flow_vs_cold=float(abs(lam - lam_c).max()))
         out["levels"].append(rec)
-        prev = (ctx, lam, U)
+        prev = (ctx, lam, U, bx)
     prev[0].close()
     out["seconds"] = time.perf_counter() - t_all
     return out
@@ -412,17 +475,17 @@ def cpu_baseline(X, V, cfg):
     import workloads
     N, b = cfg["N"], cfg["b"]
     cores = blocked.threads()
-    rows_n = int(max(16, min(N, 12.0 * cores * 2.0e7 / N)))
+    rows_n = oracle_rows_for(N, cores, 10.0)
     rows = workloads.row_sample(N, rows_n, seed=11)
     X64 = X.astype(np.float64)
     V64 = np.ascontiguousarray(V.astype(np.float64))
     w = np.full(N, 1e-2)
-    oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows[:16], w)
-    t0 = time.perf_counter()
-    oracle_step(X64, V64, cfg["beta"], cfg["alpha"], rows, w)
-    dt = time.perf_counter() - t0
-    return {"value": rows_n * float(N) * (b + 2) / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
-            "sample": f"{rows_n} sampled rows x all {N} columns, three passes (b = 1, 1, {b}), float64, rows.c + OpenMP"}
+    oracle_sample(X64, V64, cfg["beta"], rows[:16], w)
+    t_deg, t_app = oracle_sample(X64, V64, cfg["beta"], rows, w)
+    return {"value": rows_n * float(N) * b / t_app, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": t_deg + t_app,
+            "whole_step_pair_cols_per_s": rows_n * float(N) * (b + 2) / (t_deg + t_app),
+            "sample": (f"{rows_n} sampled rows x all {N} columns: block product (b = {b}) timed for the metric, the two degree "
+                       f"passes beside it; float64, rows.c + OpenMP")}
 
 
 def main():
@@ -435,14 +498,17 @@ def main():
     ap.add_argument("--path", default="", choices=["", "auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--no-eigs", action="store_true", help="skip the time-to-k-eigenpairs leg")
-    ap.add_argument("--eigs-full", action="store_true", help="also time the eigensolve at N = 2^20 (k = 128, b = 64)")
+    ap.add_argument("--no-c5-eigs", action="store_true", help="skip the eigensolve at N = 2^20 (k = 128, b = 64; about 80 s)")
+    ap.add_argument("--ladder-full", action="store_true", help="run config 5's own ladder (2^16 ... 2^20, k = 128, b = 64; many minutes)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_gpu(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    run_gpu(args)
 
 
 if __name__ == "__main__":

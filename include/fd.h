@@ -86,7 +86,7 @@ fd_status fd_destroy(fd_ctx* ctx);
  * a one-thread kernel whose bounded wait on a barrier that nothing completes must expire; the next
  * fd_synchronize then returns FD_ERR_TIMEOUT and the context stays usable).  fd_get_option also reports "last_path" (the
  * family that served the latest pass), "beta", "mean_sq", "max_sq" and "tc_cycles" (SM cycles the first CTA of the most
- * recent reduced-precision tensor-core block product spent on its work items; synchronises; with the kernel's wall time it
+ * recent tensor-core quadratic kernel spent on its work items; synchronises; with the kernel's wall time it
  * gives the SM clock the kernel actually ran at).  Unknown name -> FD_ERR_INVALID. */
 fd_status fd_set_option(fd_ctx* ctx, const char* name, double value);
 fd_status fd_get_option(const fd_ctx* ctx, const char* name, double* value_host);
@@ -229,6 +229,20 @@ fd_status fd_apply_general_static(const float* X_dev, int64_t N, int32_t D, int6
                                   const float* V_dev, int64_t ldv, int32_t b,
                                   float* Y_dev, int64_t ldy, void* cuda_stream,
                                   char* errbuf, size_t errbuf_len);
+
+/* Measured unit throughput of the GPU that is current, for the roofline of the quadratic kernels (their bound is
+ * on-chip arithmetic -- one exponential per pair, Sec. 2.2 -- not memory bandwidth, so the denominators are per-clock
+ * unit rates): exponentials (MUFU ex2), fused multiply-adds, fp32 -> packed fp16 conversions, logic and add
+ * instructions per clock per SM, and SM cycles per tcgen05.mma (kind::f16, M = 128, K = 16, fp32 accumulation) with
+ * N = 64 / 128 and the A operand in tensor memory (ts) or shared memory (ss).  Rates are counted in SM cycles, so they
+ * do not depend on the clock the GPU runs at.  scratch_dev: 256-byte aligned device buffer of at least
+ * sm_count * 4104 + 256 bytes (1 MiB is plenty), borrowed for the call.  Synchronises. */
+typedef struct {
+    int32_t sm_count;
+    double  ex2_per_clk_sm, ffma_per_clk_sm, cvt_f16x2_per_clk_sm, lop_per_clk_sm, fadd_per_clk_sm;
+    double  clk_mma_ts_n64, clk_mma_ts_n128, clk_mma_ss_n64, clk_mma_ss_n128;
+} fd_unit_rates;
+fd_status fd_unit_peaks(void* scratch_dev, size_t scratch_bytes, void* cuda_stream, fd_unit_rates* out_host);
 
 const char* fd_status_string(fd_status st);
 const char* fd_last_error(const fd_ctx* ctx);

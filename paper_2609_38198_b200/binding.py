@@ -26,13 +26,19 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
     "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_ladder_start", "fd_scale_by_degree",
-    "fd_apply_general_static", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
+    "fd_apply_general_static", "fd_unit_peaks", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
 
 class fd_eigs_info(Structure):
     _fields_ = [("applies", c_int32), ("restarts", c_int32), ("converged", c_int32), ("basis_cols", c_int32),
                 ("max_residual", c_double), ("seconds_apply", c_double), ("seconds_total", c_double)]
+
+
+class fd_unit_rates(Structure):
+    _fields_ = [("sm_count", c_int32)] + [(n, c_double) for n in (
+        "ex2_per_clk_sm", "ffma_per_clk_sm", "cvt_f16x2_per_clk_sm", "lop_per_clk_sm", "fadd_per_clk_sm",
+        "clk_mma_ts_n64", "clk_mma_ts_n128", "clk_mma_ss_n64", "clk_mma_ss_n128")]
 
 
 class fd_probe(Structure):
@@ -82,6 +88,8 @@ def _load() -> ctypes.CDLL:
     lib.fd_apply_general_static.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_double, c_void_p, c_void_p, c_void_p,
                                             c_int64, c_int32, c_void_p, c_int64, c_void_p, ctypes.c_char_p, c_size_t]
     lib.fd_apply_general_static.restype = c_int32
+    lib.fd_unit_peaks.argtypes = [c_void_p, c_size_t, c_void_p, POINTER(fd_unit_rates)]
+    lib.fd_unit_peaks.restype = c_int32
     lib.fd_status_string.argtypes = [c_int32]
     lib.fd_status_string.restype = c_char_p
     lib.fd_last_error.argtypes = [c_void_p]
@@ -296,6 +304,18 @@ def fd_apply_general_static(X: torch.Tensor, beta: float, V: torch.Tensor, left=
     if st != FD_OK:
         raise FdError(st, err.value.decode())
     return Y
+
+
+def fd_unit_peaks(device) -> dict:
+    """Measured unit throughput of `device` (fd.h: fd_unit_peaks): rates per clock per SM and SM cycles per tcgen05.mma."""
+    scratch = torch.empty(1 << 20, dtype=torch.uint8, device=device)
+    out = fd_unit_rates()
+    with torch.cuda.device(device):
+        st = lib.fd_unit_peaks(_ptr(scratch), scratch.numel(), c_void_p(torch.cuda.current_stream(device).cuda_stream),
+                               ctypes.byref(out))
+    if st != FD_OK:
+        raise FdError(st)
+    return {n: getattr(out, n) for n, _ in fd_unit_rates._fields_}
 
 
 def to_colmajor(a, device) -> torch.Tensor:

@@ -109,6 +109,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
+    const long long t_begin = clock64();
 
     // Work items of this CTA: (column chunk c, row-pair tile r) with c outermost, r = blockIdx.x + k * gridDim.x.  Every CTA
     // sweeps chunk c for all of its rows before chunk c + 1, so the whole grid reads the same L2-sized slice of the
@@ -491,6 +492,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     }
     tc_fence_before();
     __syncthreads();
+    // SM cycles CTA 0 spent on its work items (status words 2-3): lets the host relate the kernel time to the SM clock
+    if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<long long*>(p.status + 2) = clock64() - t_begin;
     if (warp == 8) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
