@@ -424,7 +424,9 @@ def time_to_k_eigs(fd, dev, args):
 
 
 def default_m_max(k, b):
-    return (max(2 * (k + 1) + b, 4 * b) + b - 1) // b * b
+    """Basis capacity for fd_eigs: room for the wanted pairs twice over plus one block, at least four blocks, and at least
+    64 columns (a very small capacity forces a thick restart on almost every step)."""
+    return (max(2 * (k + 1) + b, 4 * b, min(8 * b, 64)) + b - 1) // b * b
 
 
 def ladder(fd, dev, full=False):

@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "libfd.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC,-O3,-Wall,-Wno-unused-function", "--expt-relaxed-constexpr",
+    "-Xcompiler", "-fPIC,-O3,-Wall,-Wno-unused-function,-fopenmp", "--expt-relaxed-constexpr",
 ]
 
 
@@ -61,7 +61,7 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
             print(f"nvcc failed for {src}", file=sys.stderr)
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB, *objs]
+    link = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB, *objs, "-lgomp"]
     if verbose:
         print(" ".join(link), flush=True)
     subprocess.check_call(link)

@@ -74,7 +74,7 @@ Layout make_layout(int64_t N, int32_t D, int32_t b_max, int32_t m_max) {
         const size_t mm = (size_t)m_max * (size_t)(m_max > L.BP ? m_max : L.BP);
         size_t chunks = (size_t)ceil_div(N, 4096);
         if (chunks > 256) chunks = 256;
-        if (chunks < 2) chunks = 2;
+        if (chunks < 16) chunks = 16;     // small problems split finer so that a projection still fills the GPU
         L.eig_small_doubles = 2 * mm + chunks * mm;
         L.eig_small = carve(cur, L.eig_small_doubles * 8);
     }
@@ -133,6 +133,12 @@ fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int6
 }
 
 fd_status fd_destroy(fd_ctx* ctx) {
+    if (ctx) {
+        for (int i = 0; i < fd_ctx::kStageSlots; ++i) {
+            if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+            if (ctx->stage[i]) cudaFreeHost(ctx->stage[i]);
+        }
+    }
     delete ctx;
     return FD_OK;
 }

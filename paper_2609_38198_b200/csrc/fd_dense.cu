@@ -1,6 +1,8 @@
 // Tall-skinny dense kernels for the eigensolver (HBM-bound O(N m b) work around the quadratic
 // apply): A^T B with fp64 accumulation and a deterministic two-stage reduction, C = A S updates,
 // column copies and conversions.  All blocks are column-major with N rows.
+#include <algorithm>
+
 #include "fd_dense.h"
 
 namespace fd {
@@ -125,6 +127,30 @@ k_nn(const float* __restrict__ A, int64_t lda, int m, const float* __restrict__ 
     }
 }
 
+// out[c] = sum_i A[i, c]^2 in fp64; one block per column, fixed summation order (bit-reproducible).
+__global__ void __launch_bounds__(1024)
+k_col_sqnorms(const float* __restrict__ A, int64_t lda, int64_t N, double* __restrict__ out) {
+    __shared__ double sm[1024];
+    const float* col = A + (int64_t)blockIdx.x * lda;
+    double acc = 0.0;
+    for (int64_t i0 = 0; i0 < N; i0 += 1024 * 8) {
+        float f = 0.f;                               // 8 squares in fp32, then into the fp64 accumulator
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t i = i0 + (int64_t)u * 1024 + threadIdx.x;
+            if (i < N) { const float v = col[i]; f = fmaf(v, v, f); }
+        }
+        acc += (double)f;
+    }
+    sm[threadIdx.x] = acc;
+    __syncthreads();
+    for (int off = 512; off > 0; off >>= 1) {
+        if ((int)threadIdx.x < off) sm[threadIdx.x] += sm[threadIdx.x + off];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) out[blockIdx.x] = sm[0];
+}
+
 __global__ void k_d2f(const double* __restrict__ in, float* __restrict__ out, int64_t n, double scale) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) out[i] = (float)(in[i] * scale);
@@ -158,8 +184,12 @@ fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float
                      double* out_dev, double* scratch, size_t scratch_doubles) {
     if (m1 < 1 || m2 < 1) return FD_OK;
     const size_t mm = (size_t)m1 * m2;
-    int64_t chunks = ceil_div(N, 4096);
+    // Row chunks: at least 4096 rows each for large outputs, but enough chunks to put a few blocks on every SM when the
+    // output is small (a 32 x 32 Gram matrix is a single output tile: with 4096-row chunks it would run on 32 blocks).
+    const int64_t out_tiles = ceil_div(m1, kTnI) * ceil_div(m2, kTnJ);
+    int64_t chunks = std::max<int64_t>(ceil_div(N, 4096), ceil_div((int64_t)c->sm_count * 4, out_tiles));
     if (chunks > 256) chunks = 256;
+    if (chunks > ceil_div(N, kTnRows)) chunks = ceil_div(N, kTnRows);
     if ((size_t)chunks * mm > scratch_doubles) chunks = (int64_t)(scratch_doubles / mm);
     if (chunks < 1) return fail(c, FD_ERR_WORKSPACE, "projection scratch too small for %d x %d", m1, m2);
     int64_t rpc = round_up(ceil_div(N, chunks), kTnRows);
@@ -184,6 +214,13 @@ fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float*
         k_nn<32><<<grid, 128, 0, c->stream>>>(A, lda, m, S_dev, lds, p, C, ldc, alpha, beta, N);
     }
     FD_LAUNCH_CHECK(c, "k_nn");
+    return FD_OK;
+}
+
+fd_status col_sqnorms(fd_ctx* c, const float* A, int64_t lda, int p, int64_t N, double* out_dev) {
+    if (p < 1) return FD_OK;
+    k_col_sqnorms<<<(unsigned)p, 1024, 0, c->stream>>>(A, lda, N, out_dev);
+    FD_LAUNCH_CHECK(c, "k_col_sqnorms");
     return FD_OK;
 }
 

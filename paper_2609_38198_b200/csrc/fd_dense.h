@@ -13,6 +13,8 @@ fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float
 // C[N x p] = alpha * A[N x m] S[m x p] + beta * C; S_dev column-major floats with pitch lds.  C must not alias A.
 fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float* S_dev, int lds, int p, float* C,
                      int64_t ldc, float alpha, float beta, int64_t N);
+// out_dev[c] = |A[:, c]|^2 (fp64) for the first p columns.
+fd_status col_sqnorms(fd_ctx* c, const float* A, int64_t lda, int p, int64_t N, double* out_dev);
 fd_status d2f(fd_ctx* c, const double* in, float* out, int64_t n, double scale);
 fd_status scale_cols(fd_ctx* c, float* A, int64_t lda, int p, const float* f_dev, int64_t N);
 fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, uint32_t seed);

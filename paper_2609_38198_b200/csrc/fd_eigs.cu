@@ -41,6 +41,7 @@ struct Solver {
     double* d_scr; size_t scr_n;    // device: partials of the projections
     std::vector<double> T, G;       // host, column-major, pitch m_cap
     std::vector<double> h_out;      // host staging
+    int stage_next = 0;             // next slot of the context's pinned staging ring
     int m = 0;
     int applies = 0, restarts = 0;
     double t_apply = 0.0;
@@ -50,9 +51,26 @@ struct Solver {
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
         return FD_OK;
     }
+    // The staging ring lives in the context (pinned HOST memory, allocated once): an upload never waits for the stream
+    // unless its slot is still in flight.
+    fd_status init_staging(size_t floats) {
+        if (c->stage_floats >= floats) return FD_OK;
+        for (int i = 0; i < fd_ctx::kStageSlots; ++i) {
+            if (c->stage[i]) { FD_CUDA(c, cudaFreeHost(c->stage[i])); c->stage[i] = nullptr; }
+            FD_CUDA(c, cudaMallocHost(reinterpret_cast<void**>(&c->stage[i]), sizeof(float) * floats));
+            if (!c->stage_ev[i]) FD_CUDA(c, cudaEventCreateWithFlags(&c->stage_ev[i], cudaEventDisableTiming));
+        }
+        c->stage_floats = floats;
+        return FD_OK;
+    }
     fd_status upload_S(const std::vector<float>& S) {
-        FD_CUDA(c, cudaMemcpyAsync(d_S, S.data(), sizeof(float) * S.size(), cudaMemcpyHostToDevice, c->stream));
-        FD_CUDA(c, cudaStreamSynchronize(c->stream));      // S is a stack/vector temporary on the host
+        if (S.size() > c->stage_floats) return fail(c, FD_ERR_WORKSPACE, "staging buffer too small for a right factor");
+        const int k = stage_next;
+        stage_next = (stage_next + 1) % fd_ctx::kStageSlots;
+        FD_CUDA(c, cudaEventSynchronize(c->stage_ev[k]));  // the copy that used this slot last (four uploads ago) has finished
+        std::copy(S.begin(), S.end(), c->stage[k]);
+        FD_CUDA(c, cudaMemcpyAsync(d_S, c->stage[k], sizeof(float) * S.size(), cudaMemcpyHostToDevice, c->stream));
+        FD_CUDA(c, cudaEventRecord(c->stage_ev[k], c->stream));
         return FD_OK;
     }
 
@@ -195,6 +213,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
     S.T.assign((size_t)m_cap * m_cap, 0.0);
     S.G.assign((size_t)m_cap * m_cap, 0.0);
     S.h_out.assign((size_t)L.m_max * std::max(L.m_max, L.BP), 0.0);
+    auto t_i0 = clk::now();
+    FD_TRY(S.init_staging((size_t)L.m_max * (size_t)std::max(L.m_max, 2 * L.BP)));
+    const double t_init = secs(t_i0, clk::now());
 
     const int buffer = std::min<int>(std::min(b, 8), (int)std::max<int64_t>(0, N - nwant));
     const int nsel_max = nwant + buffer;
@@ -228,7 +249,7 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
 
     std::vector<double> theta, Xr;        // Ritz values (descending) and vectors (m x nsel, pitch m)
     std::vector<double> resid;
-    int nsel = 0, nconv = 0;
+    int nsel = 0, nconv = 0, nlock = 0;
     fd_status final_status = FD_ERR_NOT_CONVERGED;
     int stagnation = 0;
     // stagnation of the residuals at the accuracy floor of the fp32 operator (noise-smeared spectra): stop early
@@ -242,6 +263,7 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         // ---- Rayleigh-Ritz with first-order correction for G = Q^T Q = I + E ---------------------
         // Tc = T - (E T + T E) / 2 with E = G - I; T E = (E T)^T because both are symmetric
         std::vector<double> Tc((size_t)m * m), ET((size_t)m * m, 0.0);
+#pragma omp parallel for schedule(static) if (m >= 64)
         for (int j = 0; j < m; ++j)
             for (int l = 0; l < m; ++l) {
                 const double t = S.T[l + (size_t)j * m_cap];
@@ -261,6 +283,7 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         nsel = std::min(nsel_max, m);
         theta.resize(nsel);
         Xr.assign((size_t)m * nsel, 0.0);
+#pragma omp parallel for schedule(static) if (m >= 64)
         for (int jj = 0; jj < nsel; ++jj) {
             const int j = m - 1 - jj;
             theta[jj] = lam[j];
@@ -271,29 +294,45 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             }
         }
         // ---- explicit residuals R_i = W x_i - theta_i Q x_i, BP columns at a time -----------------
-        resid.assign(nsel, 0.0);
-        for (int c0 = 0; c0 < nsel; c0 += S.BP) {
-            const int w = std::min(S.BP, nsel - c0);
-            std::vector<float> Sx((size_t)m * w * 2);
-            for (int jj = 0; jj < w; ++jj)
-                for (int i = 0; i < m; ++i) {
-                    Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)(c0 + jj) * m];
-                    Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[c0 + jj] * Xr[i + (size_t)(c0 + jj) * m]);
+        // Leading pairs that converged with a margin at an earlier step are not re-evaluated every step (their Ritz
+        // vectors only improve as the basis grows); before convergence is declared every pair is evaluated afresh.
+        resid.resize(nsel, 1e300);
+        const double thr = tol * std::fabs(theta[0]);
+        bool all = false;
+        for (int pass = 0; pass < 2; ++pass) {
+            std::vector<int> act;
+            for (int i = std::min(nlock, nsel); i < nsel; ++i) act.push_back(i);
+            for (size_t a0 = 0; a0 < act.size(); a0 += (size_t)S.BP) {
+                const int w = (int)std::min<size_t>((size_t)S.BP, act.size() - a0);
+                std::vector<float> Sx((size_t)m * w * 2);
+                for (int jj = 0; jj < w; ++jj) {
+                    const int col = act[a0 + jj];
+                    for (int i = 0; i < m; ++i) {
+                        Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)col * m];
+                        Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[col] * Xr[i + (size_t)col * m]);
+                    }
                 }
-            FD_TRY(S.upload_S(Sx));
-            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
-            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
-            FD_TRY(tn_product(c, S.R, N, w, S.R, N, w, N, S.d_out, S.d_scr, S.scr_n));
-            FD_TRY(S.to_host(w * w));
-            for (int jj = 0; jj < w; ++jj) resid[c0 + jj] = std::sqrt(std::max(0.0, S.h_out[jj + (size_t)jj * w]));
+                FD_TRY(S.upload_S(Sx));
+                FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
+                FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+                FD_TRY(col_sqnorms(c, S.R, N, w, N, S.d_out));
+                FD_TRY(S.to_host(w));
+                for (int jj = 0; jj < w; ++jj) resid[act[a0 + jj]] = std::sqrt(std::max(0.0, S.h_out[jj]));
+            }
+            nconv = 0;
+            while (nconv < std::min(nwant, nsel) && resid[nconv] <= thr) ++nconv;
+            all = nsel >= nwant;
+            for (int i = 0; i < std::min(nwant, nsel); ++i) all = all && resid[i] <= thr;
+            if (all && nlock > 0) { nlock = 0; continue; }       // verify the locked pairs before declaring convergence
+            break;
+        }
+        {
+            int lead = 0;
+            while (lead < std::min(nwant, nsel) && resid[lead] <= 0.5 * thr) ++lead;
+            nlock = lead;
         }
         auto tp3 = clk::now();
         t_res += secs(tp2, tp3);
-        const double thr = tol * std::fabs(theta[0]);
-        nconv = 0;
-        while (nconv < std::min(nwant, nsel) && resid[nconv] <= thr) ++nconv;
-        bool all = nsel >= nwant;
-        for (int i = 0; i < std::min(nwant, nsel); ++i) all = all && resid[i] <= thr;
         if (all) { final_status = FD_OK; break; }
         if (S.applies >= max_applies) break;
         {
@@ -406,10 +445,11 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
     }
 #ifdef FD_EIGS_TIMING
+    fprintf(stderr, "fd_eigs: staging init %.3f s, total so far %.3f s\n", t_init, secs(t_start, clk::now()));
     fprintf(stderr, "fd_eigs: RR setup %.3f s, small eig %.3f s, residuals %.3f s, select+restart %.3f s, orthogonalise %.3f s, apply %.3f s, extend projection %.3f s\n",
             t_rr, t_eig, t_res, t_restart, t_orth, S.t_apply, t_ext);
 #else
-    (void)t_rr; (void)t_eig; (void)t_res; (void)t_restart; (void)t_orth; (void)t_ext;
+    (void)t_init; (void)t_rr; (void)t_eig; (void)t_res; (void)t_restart; (void)t_orth; (void)t_ext;
 #endif
     if (info) {
         info->applies = S.applies; info->restarts = S.restarts; info->converged = nconv; info->basis_cols = S.m;

@@ -58,6 +58,12 @@ struct fd_ctx {
     int last_path = 0;               // kernel family that served the most recent quadratic pass (FD_PATH_SIMT / FD_PATH_TC)
     double opt_tc_max_mag = 72.0;    // largest beta' * max|x - mu|^2 the Gram-form kernel is trusted with in fp32 mode
     std::string err;
+    // pinned host staging ring for the eigensolver's small uploads (allocated on the first fd_eigs, freed by fd_destroy:
+    // allocating and freeing page-locked memory on every call costs tens of milliseconds)
+    static constexpr int kStageSlots = 4;
+    float* stage[kStageSlots] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t stage_ev[kStageSlots] = {nullptr, nullptr, nullptr, nullptr};
+    size_t stage_floats = 0;
 
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
     float* xs() const { return at<float>(L.xs); }
