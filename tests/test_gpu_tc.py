@@ -311,35 +311,65 @@ def test_c4_full_size_sampled_rows(fd, dev):
     ctx.close()
 
 
-def test_c3_full_size_eigs_certificate(fd, dev):
-    """C3 at full size (N = 131072, b = 32, k = 64, beta = 2): no dense oracle is affordable, so the gates are the
-    properties that hold at any size: lambda_0 = 1 (Perron), eigenvalues in (0, 1] and descending, orthonormal vectors,
-    small residuals measured with an independent product (the direct-difference kernels), Perron vector = sqrt(d)."""
-    N, b, k, beta = 131072, 32, 64, 2.0
-    X = workloads.torus6(N, seed=42)
-    m_max = 320
+def full_size_certificate(fd, dev, X, beta, k, b, m_max, min_converged, max_applies=400, sample=256):
+    """Eigensolve at a benchmark configuration's full size, certified against the float64 oracle on sampled rows.
+
+    No dense oracle is affordable at these sizes, so the gates are (a) the properties that hold at any size -- lambda_0 = 1
+    (Perron pair, M sqrt(d) = sqrt(d)), eigenvalues in (0, 1] and descending, orthonormal vectors -- and (b) the residual
+    certificate of every returned pair from the ORACLE: rows.c evaluates (M v - theta v)_i in float64, one pair at a time,
+    on a seeded sample of rows, for all k + 1 vectors; |r| is estimated as sqrt(N / sample) |r_sample|.  For a symmetric
+    operator an eigenvalue lies within the residual norm of theta, so a pair that passes IS an eigenpair to that accuracy.
+    The scale vector s that defines M enters the oracle rows as computed on the GPU (all N values of it are needed; an
+    exact s costs two full float64 N^2 passes); it is itself checked against oracle rows here, on the same sample."""
+    from oracle import blocked
+    N = X.shape[0]
     ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=m_max)
     q, d, s, so, so2 = ctx.degree(beta, 1.0)
-    lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=300)
-    assert info.converged == k + 1
+    lam, U, info = ctx.eigs(k, b, tol=1e-6, max_applies=max_applies, allow_not_converged=True)
+    print(f"N={N} k={k} b={b}: converged {info.converged}/{k + 1} after {info.applies} applies, max residual {info.max_residual:.2e}")
+    assert info.converged >= min_converged
+    assert info.max_residual <= 2.5e-6
     assert abs(lam[0] - 1.0) <= 1e-6
-    assert np.all(np.diff(lam) <= 1e-9) and lam[-1] > 0
+    assert np.all(np.diff(lam) <= 1e-9) and lam[-1] > 0 and lam[0] <= 1.0 + 1e-6
     G = (U.double().t() @ U.double()).cpu().numpy()
     assert np.abs(G - np.eye(k + 1)).max() <= 1e-5
     sd = torch.sqrt(d.double())
     sd = sd / sd.norm()
     assert float((U[:, 0].double().abs() - sd).abs().max()) <= 1e-4 * float(sd.max())
-    # residuals with the other kernel family (degree + product on the direct-difference path)
-    ctx2 = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
-    ctx2.set_option("path", fd.FD_PATH_SIMT)
-    ctx2.degree(beta, 1.0)
-    lam_t = torch.from_numpy(lam).to(dev)
-    worst = 0.0
-    for c0 in range(0, k + 1, b):
-        blk = U[:, c0:c0 + b].t().contiguous().t()
-        MU = ctx2.apply(blk)
-        ctx2.synchronize()
-        R = MU.double() - blk.double() * lam_t[c0:c0 + b][None, :]
-        worst = max(worst, float(R.norm(dim=0).max()))
-    assert worst <= 5e-6, worst
-    ctx.close(); ctx2.close()
+    # ---- oracle rows
+    rows = workloads.row_sample(N, sample, seed=23)
+    X64 = X.astype(np.float64)
+    q64 = q.cpu().numpy().astype(np.float64)
+    s64 = s.cpu().numpy().astype(np.float64)
+    # s on the sampled rows from oracle rows of q and d (alpha = 1: d_i = q_i^-1 sum_j K_ij q_j^-1, s_i = q_i^-1 d_i^-1/2);
+    # the column vector q^-1 is the GPU's, its sampled entries are checked against the oracle first
+    q_rows = blocked.rows_apply_general(X64, beta, None, rows=rows)[:, 0]
+    assert np.abs(q64[rows] / q_rows - 1).max() <= TOL_DEG
+    d_rows = blocked.rows_apply_general(X64, beta, None, rows=rows, left=1.0 / q64, right=1.0 / q64)[:, 0]
+    s_rows = 1.0 / (q_rows * np.sqrt(d_rows))
+    assert np.abs(s64[rows] / s_rows - 1).max() <= TOL_DEG
+    U64 = np.ascontiguousarray(U.cpu().numpy().astype(np.float64))
+    MU = blocked.rows_apply_general(X64, beta, U64, rows=rows, left=s64, right=s64)
+    R = MU - U64[rows] * lam[None, :]
+    est = np.sqrt(N / float(sample)) * np.linalg.norm(R, axis=0)
+    print(f"   oracle-row residual estimates: max {est.max():.2e}, median {np.median(est):.2e}")
+    assert est.max() <= 7.5e-6, est.max()          # the 5e-6 certificate with room for the sampling error of 256 rows
+    ctx.close()
+    return lam, info
+
+
+def test_c3_full_size_eigs_certificate(fd, dev):
+    """C3 at full size: N = 131072, b = 32, k = 64, beta = 2."""
+    full_size_certificate(fd, dev, workloads.torus6(131072, seed=42), 2.0, 64, 32, 192, min_converged=65)
+
+
+def test_c4_full_size_eigs_certificate(fd, dev):
+    """C4 at full size: N = 262144, D = 30 (tensor-core distance), b = 32, k = 32, beta = 2."""
+    full_size_certificate(fd, dev, workloads.latent_torus(262144, seed=42), 2.0, 32, 32, 128, min_converged=33)
+
+
+def test_c5_full_size_eigs_certificate(fd, dev):
+    """C5 at full size: N = 2^20, b = 64, k = 128, beta = 2.  k = 128 cuts the third cluster of the 6-torus spectrum
+    (multiplicities 1 + 12 + 60 = 73, then 160): the pairs inside the cut cluster stall just above tol = 1e-6 at the fp32
+    operator's residual floor, which is a reported outcome; all 129 pairs must pass the oracle-row certificate."""
+    full_size_certificate(fd, dev, workloads.torus6(1 << 20, seed=42), 2.0, 128, 64, 384, min_converged=73, sample=128)
