@@ -35,8 +35,8 @@ METRIC = "kernel-apply pair-columns per second of the block product Y = M V (N^2
 UNIT = "pair*cols/s"
 
 # DRAM bytes per launch of the timed block-product kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture at N = 2^20, summarised under profiles/), keyed by the kernel that bench times; None = not captured.
-NCU_TRAFFIC_BYTES = {"k_tc<64, block>": None, "k_simt": None}
+# capture of this kernel at N = 2^20, single-pass metrics), keyed by the kernel that bench times; None = not captured.
+NCU_TRAFFIC_BYTES = {"k_tc<64, block>": 25.015e9 + 2.181e9, "k_simt": None}
 
 
 def measured_peaks():
@@ -242,12 +242,15 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
+    # the clock sampler starts before the warm-up (nvidia-smi's own start-up can stall the GPU for a moment); only the
+    # samples taken during the timed region are kept
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler.lines.clear()
     timers = []
     launches0 = fd.fd_launch_count()
     t_start, t_end = ev(), ev()
@@ -264,13 +267,27 @@ def run_gpu(args):
     app_ms = float(np.mean([b_.elapsed_time(c_) for _, b_, c_ in timers]))
     path_used = "tc" if ctx.get_option("last_path") == 2 else "simt"
 
-    # SM clock the block-product kernel actually ran at: SM cycles of its first CTA over the kernel's duration
-    sustained_mhz = None
+    # SM clock the block-product kernel actually runs at (it draws the board's power limit, so the clock sags): median of
+    # nvidia-smi samples over a loop of block products alone, and, as a cross-check from the kernel itself, the SM cycles
+    # its first CTA counted over the kernel's duration (a lower bound: the count excludes launch and tail)
+    sustained_mhz = cycles_mhz = None
     if path_used == "tc":
+        s2 = ClockSampler(local)
+        if rank == 0:
+            s2.start()
+            time.sleep(0.5)
+            s2.lines.clear()
         e0, e1 = ev(), ev()
-        e0.record(stream); ctx.apply(Vd, out=Yd); e1.record(stream)
+        reps = max(4, int(2000.0 / max(app_ms, 1.0)))
+        e0.record(stream)
+        for _ in range(min(reps, 50)):
+            ctx.apply(Vd, out=Yd)
+        e1.record(stream)
         torch.cuda.synchronize(dev)
-        sustained_mhz = ctx.get_option("tc_cycles") / (e0.elapsed_time(e1) * 1e3)
+        if rank == 0:
+            c2 = s2.stop()
+            sustained_mhz = c2.get("sm_mhz")
+        cycles_mhz = ctx.get_option("tc_cycles") / (e0.elapsed_time(e1) / min(reps, 50) * 1e3)
     # the reduced-precision product, reported separately (three repeats)
     fast_ms = None
     if path_used == "tc":
@@ -332,7 +349,7 @@ def run_gpu(args):
                     "frac": pairs_per_s / peak_pairs,
                     "peak_source": (f"measured unit rate ({rates['ex2_per_clk_sm']:.2f} ex2/clk/SM, {rates['sm_count']} SMs; "
                                     f"fd_unit_peaks in this run) x maximum SM clock {sm_max:.0f} MHz ({peak_kind})"),
-                    "sustained_sm_mhz": sustained_mhz,
+                    "sustained_sm_mhz": sustained_mhz, "sm_mhz_from_kernel_cycles": cycles_mhz,
                     "frac_at_sustained_clock": (pairs_per_s / (peak_pairs * sustained_mhz / sm_max)) if sustained_mhz else None,
                     "traffic": NCU_TRAFFIC_BYTES.get(kernel_name) if N == (1 << 20) else None,
                     "algorithmic_bytes": 4.0 * N * (D + 2 * b + 2),
@@ -387,6 +404,15 @@ def time_to_k_eigs(fd, dev, args):
              ("C4 latent torus R^30", workloads.latent_torus(262144, seed=42), 32, 32, 2.0, 600)]
     if not args.no_c5_eigs:
         cases.append(("C5 6-torus", workloads.torus6(1 << 20, seed=42), 128, 64, 2.0, 400))
+    if args.eigs_case:
+        # restrict the leg to one configuration (for profiling a single solve); C2 keeps its four bandwidths
+        pts = None
+        picked = []
+        for cse in cases:
+            pts = cse[1] if cse[1] is not None else pts
+            if cse[0].startswith(args.eigs_case):
+                picked.append((cse[0], pts) + cse[2:])
+        cases = picked
     Xnp = None
     for name, Xc, k, b, beta, max_applies in cases:
         if Xc is not None:
@@ -419,7 +445,8 @@ def time_to_k_eigs(fd, dev, args):
         del ctx, X
         torch.cuda.empty_cache()
         res.append(rec)
-    res.append(ladder(fd, dev, args.ladder_full))
+    if not args.eigs_case:
+        res.append(ladder(fd, dev, args.ladder_full))
     return res
 
 
@@ -501,6 +528,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--no-eigs", action="store_true", help="skip the time-to-k-eigenpairs leg")
     ap.add_argument("--no-c5-eigs", action="store_true", help="skip the eigensolve at N = 2^20 (k = 128, b = 64; about 80 s)")
+    ap.add_argument("--eigs-case", default="", choices=["", "C1", "C2", "C3", "C4", "C5"],
+                    help="time-to-k-eigenpairs leg: only this configuration (and no ladder)")
     ap.add_argument("--ladder-full", action="store_true", help="run config 5's own ladder (2^16 ... 2^20, k = 128, b = 64; many minutes)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -65,6 +65,11 @@ typedef enum {
 /* Which kernel family serves the quadratic passes (fd_set_option "path"). */
 enum { FD_PATH_AUTO = 0, FD_PATH_SIMT = 1, FD_PATH_TC = 2 };
 
+/* Largest number of coordinates per point the kernels cover: D <= 32 on both kernel families, 33..FD_MAX_D on the
+ * Gram-form tensor-core family only (a pass whose bandwidth exceeds that family's accuracy budget, beta * log2(e) *
+ * max|x - mu|^2 >= "tc_max_mag", then returns FD_ERR_UNSUPPORTED).  fd_create refuses D > FD_MAX_D. */
+#define FD_MAX_D 60
+
 /* Bytes of device workspace fd_create needs.  O(N (D + b_max + m_max)); no N^2 term.
  * b_max: widest block passed to fd_apply / fd_apply_general (1..256).
  * m_max: basis capacity for fd_eigs (columns); 0 if fd_eigs will not be called. */

@@ -101,7 +101,7 @@ using namespace fd;
 extern "C" {
 
 size_t fd_workspace_bytes(int64_t N, int32_t D, int32_t b_max, int32_t m_max) {
-    if (N < 1 || D < 1 || b_max < 1 || b_max > 256 || m_max < 0) return 0;
+    if (N < 1 || D < 1 || D > FD_MAX_D || b_max < 1 || b_max > 256 || m_max < 0) return 0;
     return make_layout(N, D, b_max, m_max).total;
 }
 
@@ -109,8 +109,9 @@ fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int6
                     int32_t b_max, int32_t m_max, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
     if (!out) return FD_ERR_INVALID;
     *out = nullptr;
-    if (!X_dev || !ws_dev || N < 1 || D < 1 || D > 512 || ldx < D || b_max < 1 || b_max > 256 || m_max < 0)
+    if (!X_dev || !ws_dev || N < 1 || D < 1 || ldx < D || b_max < 1 || b_max > 256 || m_max < 0)
         return FD_ERR_INVALID;
+    if (D > FD_MAX_D) return FD_ERR_UNSUPPORTED;                 // no kernel covers more coordinates
     if (N > ((int64_t)1 << 31) - 1024) return FD_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(ws_dev) & 255) != 0) return FD_ERR_INVALID;
     Layout L = make_layout(N, D, b_max, m_max);
@@ -247,6 +248,16 @@ static fd_status check_block(fd_ctx* c, const float* p, int64_t ld, int64_t rows
 fd_status fd_apply_general(fd_ctx* c, double beta, const float* left_dev, const float* right_dev,
                            const float* Xrow_dev, int64_t Nrow, int64_t ldxrow, const float* V_dev, int64_t ldv,
                            int32_t b, float* Y_dev, int64_t ldy, fd_precision prec) {
+    return fd::apply_general(c, beta, left_dev, right_dev, false, Xrow_dev, Nrow, ldxrow, V_dev, ldv, b, Y_dev, ldy, prec);
+}
+
+}  // extern "C"
+
+namespace fd {
+
+fd_status apply_general(fd_ctx* c, double beta, const float* left_dev, const float* right_dev, bool right_pos,
+                        const float* Xrow_dev, int64_t Nrow, int64_t ldxrow, const float* V_dev, int64_t ldv, int32_t b,
+                        float* Y_dev, int64_t ldy, fd_precision prec) {
     if (!c) return FD_ERR_INVALID;
     if (!(beta > 0) || !(beta < 1e30)) return fail(c, FD_ERR_INVALID, "beta out of range");
     if (prec != FD_PREC_FP32 && prec != FD_PREC_FAST) return fail(c, FD_ERR_INVALID, "bad precision");
@@ -272,6 +283,7 @@ fd_status fd_apply_general(fd_ctx* c, double beta, const float* left_dev, const 
     }
     ApplyArgs a{};
     a.beta = beta; a.right = right_dev; a.V = V_dev; a.ldv = ldv; a.b = b; a.prec = prec; a.rowsq = nullptr;
+    a.right_pos = right_pos;
     if (!Xrow_dev) {
         a.xrow = c->xs(); a.Nrow = N; a.rows_are_ctx = true; a.left = left_dev; a.Y = Y_dev; a.ldy = ldy;
         return apply_dispatch(c, a);
@@ -286,6 +298,10 @@ fd_status fd_apply_general(fd_ctx* c, double beta, const float* left_dev, const 
     }
     return FD_OK;
 }
+
+}  // namespace fd
+
+extern "C" {
 
 fd_status fd_apply(fd_ctx* c, const float* V_dev, int64_t ldv, int32_t b, float* Y_dev, int64_t ldy, fd_precision prec) {
     if (!c) return FD_ERR_INVALID;

@@ -161,7 +161,8 @@ extern "C" fd_status fd_nystrom(fd_ctx* c, const float* Xnew_dev, int64_t Nnew, 
     for (int64_t r0 = 0; r0 < Nnew; r0 += N) {
         const int64_t n = std::min(N, Nnew - r0);
         const float* xr = Xnew_dev + r0 * ldxnew;
-        FD_TRY(fd_apply_general(c, c->beta, nullptr, c->w(), xr, n, ldxnew, nullptr, N, 1, den, n, FD_PREC_FP32));
+        // the denominator's right vector q^-alpha is positive: it may take the same kernel family as the numerators
+        FD_TRY(apply_general(c, c->beta, nullptr, c->w(), true, xr, n, ldxnew, nullptr, N, 1, den, n, FD_PREC_FP32));
         for (int c0 = 0; c0 < m; c0 += c->L.b_max) {
             const int w = std::min<int>(c->L.b_max, m - c0);
             FD_TRY(fd_apply_general(c, c->beta, nullptr, c->w(), xr, n, ldxnew, psi_dev + (int64_t)c0 * ldpsi, ldpsi, w,

@@ -46,6 +46,7 @@ struct fd_ctx {
     int centered = 0;
     double mean_sq = 0.0;            // N^-1 sum |x_i - mu|^2 (Eq. 7)
     double max_sq = 0.0;             // max_i |x_i - mu|^2
+    double row_max_sq = 0.0;         // the same maximum over the external rows staged most recently (rectangular products)
     // current operator state (set by fd_degree)
     bool have_s = false;
     double beta = 0.0, alpha = 0.0;
@@ -121,6 +122,11 @@ fd_status apply_simt(fd_ctx* c, const ApplyArgs& a);
 fd_status apply_tc(fd_ctx* c, const ApplyArgs& a);
 bool tc_supported(const fd_ctx* c, const ApplyArgs& a);
 fd_status apply_dispatch(fd_ctx* c, const ApplyArgs& a);
+// Body of fd_apply_general with one more promise: right_pos = the caller guarantees right > 0 elementwise, which lets a
+// row-sum (V == nullptr) with a right vector take the same kernel family as the block products of the same operator.
+fd_status apply_general(fd_ctx* c, double beta, const float* left_dev, const float* right_dev, bool right_pos,
+                        const float* Xrow_dev, int64_t Nrow, int64_t ldxrow, const float* V_dev, int64_t ldv, int32_t b,
+                        float* Y_dev, int64_t ldy, fd_precision prec);
 // Reads and clears the tensor-core kernel's status word; FD_ERR_TIMEOUT if a bounded wait expired.  Synchronises.
 fd_status tc_check_status(fd_ctx* c);
 // Launches a one-thread kernel whose bounded wait must expire after limit_cycles (test of the time-out plumbing).

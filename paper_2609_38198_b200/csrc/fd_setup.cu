@@ -165,6 +165,19 @@ fd_status stage_rows(fd_ctx* c, const float* Xrow_dev, int64_t ldxrow, int64_t r
     k_pad_copy<<<grid_for(n * L.DP, 256, 148 * 16), 256, 0, c->stream>>>(Xrow_dev + r0 * ldxrow, ldxrow, n, L.D, L.DP,
                                                                          c->at<float>(L.xrow));
     FD_LAUNCH_CHECK(c, "k_pad_copy(rows)");
+    // largest |x - mu|^2 among the staged rows: the Gram-form kernel's exponent budget must hold for them too, and
+    // external rows may lie further from the centre than any of the context's own points (scratch: split partials)
+    double* part = c->at<double>(L.part);
+    const int nb = grid_for(n, 256, 512);
+    k_sqnorm_partial<<<nb, 256, 0, c->stream>>>(c->at<float>(L.xrow), n, L.DP, c->at<double>(L.mu), part, part + 1024);
+    FD_LAUNCH_CHECK(c, "k_sqnorm_partial(rows)");
+    double host[2048];
+    FD_CUDA(c, cudaMemcpyAsync(host, part, sizeof(double) * 2048, cudaMemcpyDeviceToHost, c->stream));
+    FD_CUDA(c, cudaStreamSynchronize(c->stream));
+    double tot = 0.0, mx = 0.0;
+    for (int i = 0; i < nb; ++i) { tot += host[i]; if (host[1024 + i] > mx) mx = host[1024 + i]; }
+    if (!(tot == tot) || !(tot < 1e300)) return fail(c, FD_ERR_NONFINITE, "non-finite row points");
+    c->row_max_sq = mx;
     return FD_OK;
 }
 

@@ -674,10 +674,11 @@ bool tc_supported(const fd_ctx* c, const ApplyArgs& a) {
     // The decision depends only on the data set, the bandwidth and the precision mode -- never on the kind of pass --
     // so the degree passes and the block products of one operator always run on the same kernel family (their
     // common rounding bias then cancels in diag(s) K diag(s)).
-    if (c->opt_path != FD_PATH_TC && L.N < 16384) return false;    // small problems: the split direct-difference kernel fills the GPU better
+    // small problems: the split direct-difference kernel fills the GPU better (it covers D <= 32 only)
+    if (c->opt_path != FD_PATH_TC && L.N < 16384 && L.DP <= 32) return false;
     const double bprime = a.beta * kLog2e;
     // exponent magnitude the fp16 hi/lo norm pieces and the fp32 Gram accumulation can carry accurately
-    const double mag = bprime * c->max_sq;
+    const double mag = bprime * (a.rows_are_ctx ? c->max_sq : std::max(c->max_sq, c->row_max_sq));
     if (!(mag < (a.prec == FD_PREC_FAST ? 2000.0 : c->opt_tc_max_mag))) return false;
     if (a.V == nullptr && a.right != nullptr && !a.right_pos) return false;   // row-sum mode folds a POSITIVE right vector into e_j
     return true;

@@ -252,6 +252,29 @@ def test_nystrom_matches_oracle_and_reproduces_samples(fd, dev):
     ctx.close()
 
 
+def test_nystrom_on_the_automatic_path_at_n16384(fd, dev):
+    """N = 16384 is where the automatic choice hands the kernel sums to the Gram-form tensor-core family: the
+    extension (a rectangular numerator product and a row-sum denominator with a positive right vector) must stay
+    on it and match the formula.  The extended functions are smooth test functions, not eigenvectors: the formula
+    does not care, and no 16384^3 eigensolve is needed."""
+    N, beta, alpha = 16384, 3.0, 1.0
+    X = workloads.torus6(N, seed=21)
+    Z = workloads.torus6(1500, seed=22)
+    rng = np.random.default_rng(5)
+    A = rng.standard_normal((X.shape[1], 5))
+    psi = np.cos(X.astype(np.float64) @ A) + 0.25
+    lam = np.array([1.0, 0.9, 0.8, 0.55, 0.3])
+    q_o = dense.degree(X, beta, alpha)[0]
+    ext_o = nystrom.extend(X, q_o, alpha, beta, psi, lam, Z)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8)                  # path: automatic
+    ctx.degree(beta, alpha)
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    ext = ctx.nystrom(torch.from_numpy(Z).to(dev), fd.to_colmajor(psi, dev), lam).cpu().numpy()
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    assert np.abs(ext - ext_o).max() <= 2e-5 * np.abs(ext_o).max()
+    ctx.close()
+
+
 def test_ladder_start_matches_oracle_and_warm_solve(fd, dev):
     """One rung of the (n, beta) ladder: eigenpairs on the first 2500 points -> start basis on 5000 points.
     Inputs to the extension (eigenvectors, eigenvalues) come from the oracle; the GPU and the oracle both extend them.

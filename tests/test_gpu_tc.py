@@ -78,6 +78,38 @@ def test_dimensions_and_k_slabs(fd, dev, D, beta):
     tc_case(fd, dev, X, beta, 1.0, 32)
 
 
+def test_dimensions_33_to_60_take_the_gram_form_path_at_any_size(fd, dev):
+    # 32 < D <= 60 is covered by the tensor-core family alone: the automatic choice must pick it even for a small point
+    # set, and a bandwidth beyond its accuracy budget is refused instead of silently served by nothing
+    X = workloads.latent_torus(2000, seed=40, D=40)
+    V = workloads.block(2000, 16, seed=4)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=16)            # path: automatic
+    q, d, s, so, so2 = ctx.degree(0.5, 1.0)
+    Y = ctx.apply(fd.to_colmajor(V, dev))
+    ctx.synchronize()
+    assert ctx.get_option("last_path") == fd.FD_PATH_TC
+    assert relF(Y.cpu().numpy(), dense.apply(X, 0.5, 1.0, V)) <= TOL_APPLY
+    with pytest.raises(fd.FdError) as e:
+        ctx.degree(500.0, 1.0)
+    assert e.value.status == fd.FD_ERR_UNSUPPORTED
+    ctx.close()
+    assert fd.fd_workspace_bytes(64, 61, 8, 32) == 0                   # D > FD_MAX_D: no workspace size, no context
+    with pytest.raises(fd.FdError):
+        fd.Context(torch.zeros((64, 61), dtype=torch.float32, device=dev), b_max=8)
+
+
+def test_non_finite_points_are_refused(fd, dev):
+    X = workloads.torus6(500, seed=1)
+    X[123, 4] = np.nan
+    with pytest.raises(fd.FdError) as e:
+        fd.Context(torch.from_numpy(X).to(dev), b_max=8)
+    assert e.value.status == fd.FD_ERR_NONFINITE
+    X[123, 4] = np.inf
+    with pytest.raises(fd.FdError) as e:
+        fd.Context(torch.from_numpy(X).to(dev), b_max=8)
+    assert e.value.status == fd.FD_ERR_NONFINITE
+
+
 @pytest.mark.parametrize("alpha", [0.0, 0.5, 1.0])
 def test_alpha(fd, dev, alpha):
     tc_case(fd, dev, workloads.torus6(1500, seed=4), 1.5, alpha, 32)
