@@ -54,7 +54,8 @@ typedef enum {
     FD_ERR_PERRON_WALL = 5,    /* Eq. 12 failed: g_P <= kappa_P * eta                          */
     FD_ERR_UNSUPPORTED = 6,    /* shape outside what the kernels cover                         */
     FD_ERR_TIMEOUT = 7,        /* a bounded device-side wait expired (status word set)         */
-    FD_ERR_NONFINITE = 8       /* non-finite input or intermediate detected                    */
+    FD_ERR_NONFINITE = 8,      /* non-finite input or intermediate detected                    */
+    FD_ERR_COMM = 9            /* an exchange callback of a row-sharded context reported failure */
 } fd_status;
 
 typedef enum {
@@ -207,6 +208,46 @@ fd_status fd_ladder_start(fd_ctx* old_level, fd_ctx* new_level, const float* Xne
  * context's current d (power = -0.5: Markov right eigenvectors from symmetric ones). */
 fd_status fd_scale_by_degree(fd_ctx* ctx, const float* v_dev, int64_t ldv, int32_t cols,
                              double power, float* out_dev, int64_t ldout);
+
+/* ---- Row-sharded operation: several processes, one GPU each (Sec. 3: multi-GPU runs are sharded over the row axis) ----
+ *
+ * Every rank creates its context on ALL N points (N D floats: tens of megabytes at most) and owns the rows
+ * [row_begin, row_end) that fd_shard_rows assigns: `world` contiguous ranges of round_up(ceil(N / world), 256) rows,
+ * the last ones shorter or empty.  Once fd_set_shard has been called,
+ *   - every quadratic pass evaluates the owned rows only (N / world rows against all N columns);
+ *   - fd_degree exchanges q and d (one column each) and sums its two scalars over the ranks;
+ *   - fd_apply / fd_apply_general (square form) exchange the rows of Y, so Y is complete on every rank on return;
+ *   - fd_eigs keeps the basis, its image and every tall-skinny product on the owned rows; per expansion it
+ *     exchanges the rows of the new N x b block before the product and sums the small projected matrices over
+ *     the ranks on the host; eigenvector outputs are complete on every rank; fd_beta_flow inherits all of this;
+ *   - rectangular products (external rows), fd_nystrom and fd_ladder_start stay replicated: each rank computes all.
+ * All ranks must make the same calls in the same order with the same arguments (the usual collective rule); the
+ * host-side decisions of fd_eigs and fd_beta_flow depend only on summed quantities, which the callbacks must return
+ * bit-identical on every rank (NCCL, gloo and MPI all-reduce do).
+ *
+ * The library links no communication library: the caller supplies two callbacks (torch.distributed / NCCL in the
+ * Python binding) and the exchange buffer.
+ *   allreduce_sum_host(user, buf, n): in-place sum over the ranks of n host doubles; blocking.
+ *   allgather_dev(user, send_dev, recv_dev, count): every rank contributes count floats at send_dev; on return
+ *     recv_dev holds world * count floats ordered by rank.  The callback is called with all earlier work of the
+ *     context enqueued on the context's stream and must order itself after that work and before anything enqueued
+ *     on that stream afterwards (a collective enqueued on that stream, or one that synchronises on both sides).
+ *     send_dev and recv_dev lie inside xchg_dev.
+ * Both return 0 on success; anything else makes the current call return FD_ERR_COMM.
+ * xchg_dev: device buffer of at least fd_shard_exchange_bytes(N, b_max, world) bytes, 256-byte aligned, borrowed
+ * until fd_destroy or fd_set_shard(ctx, NULL).  fd_set_shard(ctx, NULL) returns the context to unsharded operation. */
+typedef struct {
+    int32_t rank, world;
+    int (*allreduce_sum_host)(void* user, double* buf, int64_t n);
+    int (*allgather_dev)(void* user, const float* send_dev, float* recv_dev, int64_t count);
+    void*   user;
+    void*   xchg_dev;
+    size_t  xchg_bytes;
+} fd_shard;
+/* Pure host arithmetic, no GPU needed. */
+fd_status fd_shard_rows(int64_t N, int32_t world, int32_t rank, int64_t* row_begin, int64_t* row_end);
+size_t    fd_shard_exchange_bytes(int64_t N, int32_t b_max, int32_t world);
+fd_status fd_set_shard(fd_ctx* ctx, const fd_shard* shard);
 
 /* No counterpart in the paper: an entry point for callers that cannot allocate device memory.
  *

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfd.so")
 
 FD_OK, FD_ERR_INVALID, FD_ERR_WORKSPACE, FD_ERR_CUDA, FD_ERR_NOT_CONVERGED = 0, 1, 2, 3, 4
-FD_ERR_PERRON_WALL, FD_ERR_UNSUPPORTED, FD_ERR_TIMEOUT, FD_ERR_NONFINITE = 5, 6, 7, 8
+FD_ERR_PERRON_WALL, FD_ERR_UNSUPPORTED, FD_ERR_TIMEOUT, FD_ERR_NONFINITE, FD_ERR_COMM = 5, 6, 7, 8, 9
 FD_PREC_FP32, FD_PREC_FAST = 0, 1
 FD_PATH_AUTO, FD_PATH_SIMT, FD_PATH_TC = 0, 1, 2
 FD_FLOW_VERTEX, FD_FLOW_PERRON_WALL, FD_FLOW_LEFT_EDGE, FD_FLOW_RIGHT_EDGE = 0, 1, 2, 3
@@ -26,7 +26,7 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
     "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_ladder_start", "fd_scale_by_degree",
-    "fd_apply_general_static", "fd_unit_peaks", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
+    "fd_apply_general_static", "fd_unit_peaks", "fd_shard_rows", "fd_shard_exchange_bytes", "fd_set_shard", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
 
@@ -174,8 +174,20 @@ class Context:
 
     def _check(self, st: int, ok=(FD_OK,)):
         if st not in ok:
+            shard = getattr(self, "_shard", None)
+            if st == FD_ERR_COMM and shard is not None and shard.error is not None:
+                err, shard.error = shard.error, None
+                raise FdError(st, lib.fd_last_error(self._h).decode()) from err
             raise FdError(st, lib.fd_last_error(self._h).decode())
         return st
+
+    def set_shard(self, shard):
+        """Row-sharded operation (fd_set_shard): `shard` is a shard.Shard built for this context's (N, b_max), or
+        None to return to unsharded operation.  The context keeps the shard (buffer and callbacks) alive."""
+        if shard is not None:
+            assert shard.N == self.N and shard.b_max >= self.b_max
+        self._check(lib.fd_set_shard(self._h, ctypes.byref(shard.struct) if shard is not None else None))
+        self._shard = shard
 
     def set_option(self, name: str, value: float):
         self._check(lib.fd_set_option(self._h, name.encode(), float(value)))

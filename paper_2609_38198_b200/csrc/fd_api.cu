@@ -207,13 +207,18 @@ fd_status fd_degree(fd_ctx* c, double beta, double alpha, fd_precision prec, flo
     c->have_s = false;
     double* rowsq = c->at<double>(c->L.rowsq);
     // pass 1: q = K 1 (and sum_j K_ij^2 per row)
+    // (the rows this rank owns: all of them unless the context is row-sharded)
+    const int64_t r0 = c->row0(), n = c->rows();
     ApplyArgs a{};
-    a.xrow = c->xs(); a.Nrow = N; a.rows_are_ctx = true; a.beta = beta;
+    a.xrow = c->xs() + r0 * c->L.DP; a.Nrow = n; a.rows_are_ctx = true; a.beta = beta;
     a.left = nullptr; a.right = nullptr; a.V = nullptr; a.ldv = N; a.b = 1;
-    a.Y = c->q(); a.ldy = N; a.rowsq = rowsq; a.prec = prec;
-    FD_TRY(apply_dispatch(c, a));
-    double sum_q = 0, sum_sq = 0;
-    FD_TRY(reduce_sums(c, c->q(), rowsq, N, &sum_q, &sum_sq));
+    a.Y = c->q() + r0; a.ldy = N; a.rowsq = rowsq + r0; a.prec = prec;
+    if (n > 0) FD_TRY(apply_dispatch(c, a));
+    double sums[2] = {0.0, 0.0};
+    if (n > 0) FD_TRY(reduce_sums(c, c->q() + r0, rowsq + r0, n, &sums[0], &sums[1]));
+    FD_TRY(allreduce_host(c, sums, 2));
+    FD_TRY(gather_rows(c, c->q(), N, 1));
+    const double sum_q = sums[0], sum_sq = sums[1];
     if (!(sum_q == sum_q) || !(sum_q < 1e300)) return fail(c, FD_ERR_NONFINITE, "non-finite degree sum");
     if (alpha == 0.0) {
         // d = q, s = q^-1/2
@@ -223,8 +228,9 @@ fd_status fd_degree(fd_ctx* c, double beta, double alpha, fd_precision prec, flo
         // pass 2: d = q^-alpha * K q^-alpha
         FD_TRY(ew_pow(c, c->q(), -alpha, c->w(), N));
         ApplyArgs a2 = a;
-        a2.left = c->w(); a2.right = c->w(); a2.Y = c->d(); a2.rowsq = nullptr; a2.right_pos = true;
-        FD_TRY(apply_dispatch(c, a2));
+        a2.left = c->w() + r0; a2.right = c->w(); a2.Y = c->d() + r0; a2.rowsq = nullptr; a2.right_pos = true;
+        if (n > 0) FD_TRY(apply_dispatch(c, a2));
+        FD_TRY(gather_rows(c, c->d(), N, 1));
         FD_TRY(ew_scale_vec(c, c->w(), c->d(), c->s(), N));
     }
     if (q_dev) FD_CUDA(c, cudaMemcpyAsync(q_dev, c->q(), (size_t)N * 4, cudaMemcpyDeviceToDevice, c->stream));
@@ -257,7 +263,7 @@ namespace fd {
 
 fd_status apply_general(fd_ctx* c, double beta, const float* left_dev, const float* right_dev, bool right_pos,
                         const float* Xrow_dev, int64_t Nrow, int64_t ldxrow, const float* V_dev, int64_t ldv, int32_t b,
-                        float* Y_dev, int64_t ldy, fd_precision prec) {
+                        float* Y_dev, int64_t ldy, fd_precision prec, bool gather_out) {
     if (!c) return FD_ERR_INVALID;
     if (!(beta > 0) || !(beta < 1e30)) return fail(c, FD_ERR_INVALID, "beta out of range");
     if (prec != FD_PREC_FP32 && prec != FD_PREC_FAST) return fail(c, FD_ERR_INVALID, "bad precision");
@@ -285,8 +291,13 @@ fd_status apply_general(fd_ctx* c, double beta, const float* left_dev, const flo
     a.beta = beta; a.right = right_dev; a.V = V_dev; a.ldv = ldv; a.b = b; a.prec = prec; a.rowsq = nullptr;
     a.right_pos = right_pos;
     if (!Xrow_dev) {
-        a.xrow = c->xs(); a.Nrow = N; a.rows_are_ctx = true; a.left = left_dev; a.Y = Y_dev; a.ldy = ldy;
-        return apply_dispatch(c, a);
+        // square product: the rows this rank owns (all of them unless the context is row-sharded)
+        const int64_t r0 = c->row0(), n = c->rows();
+        a.xrow = c->xs() + r0 * c->L.DP; a.Nrow = n; a.rows_are_ctx = true;
+        a.left = left_dev ? left_dev + r0 : nullptr; a.Y = Y_dev + r0; a.ldy = ldy;
+        if (n > 0) FD_TRY(apply_dispatch(c, a));
+        if (gather_out) FD_TRY(gather_rows(c, Y_dev, ldy, b));
+        return FD_OK;
     }
     // rectangular product: stage the external rows chunk by chunk through the row scratch
     for (int64_t r0 = 0; r0 < Nrow; r0 += N) {
@@ -336,6 +347,7 @@ const char* fd_status_string(fd_status st) {
         case FD_ERR_UNSUPPORTED: return "unsupported shape";
         case FD_ERR_TIMEOUT: return "bounded device wait expired";
         case FD_ERR_NONFINITE: return "non-finite value";
+        case FD_ERR_COMM: return "exchange callback of a row-sharded context failed";
     }
     return "unknown status";
 }

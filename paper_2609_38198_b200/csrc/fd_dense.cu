@@ -163,11 +163,11 @@ __global__ void k_scale_cols(float* __restrict__ A, int64_t lda, int p, const fl
 }
 
 // Counter-based uniform(-1, 1) fill for cold-start blocks (hash of (seed, element index)).
-__global__ void k_random_fill(float* __restrict__ A, int64_t lda, int p, int64_t N, uint32_t seed) {
+__global__ void k_random_fill(float* __restrict__ A, int64_t lda, int p, int64_t N, int64_t row0, uint32_t seed) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     for (int c = 0; c < p; ++c) {
-        uint64_t z = (uint64_t)i * 0x9E3779B97F4A7C15ull + ((uint64_t)(c + 1) << 40) + seed;
+        uint64_t z = (uint64_t)(i + row0) * 0x9E3779B97F4A7C15ull + ((uint64_t)(c + 1) << 40) + seed;
         z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
         A[i + (int64_t)c * lda] = (float)((double)(z >> 11) * (2.0 / 9007199254740992.0) - 1.0);
     }
@@ -184,6 +184,10 @@ fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float
                      double* out_dev, double* scratch, size_t scratch_doubles) {
     if (m1 < 1 || m2 < 1) return FD_OK;
     const size_t mm = (size_t)m1 * m2;
+    if (N < 1) {                                                  // a rank that owns no rows contributes zeros
+        FD_CUDA(c, cudaMemsetAsync(out_dev, 0, mm * sizeof(double), c->stream));
+        return FD_OK;
+    }
     // Row chunks: at least 4096 rows each for large outputs, but enough chunks to put a few blocks on every SM when the
     // output is small (a 32 x 32 Gram matrix is a single output tile: with 4096-row chunks it would run on 32 blocks).
     const int64_t out_tiles = ceil_div(m1, kTnI) * ceil_div(m2, kTnJ);
@@ -204,7 +208,7 @@ fd_status tn_product(fd_ctx* c, const float* A, int64_t lda, int m1, const float
 
 fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float* S_dev, int lds, int p, float* C,
                      int64_t ldc, float alpha, float beta, int64_t N) {
-    if (p < 1) return FD_OK;
+    if (p < 1 || N < 1) return FD_OK;
     if (m < 1) return fail(c, FD_ERR_INVALID, "nn_product: m < 1");
     if (p <= 8) {
         dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(p, 8));
@@ -219,6 +223,10 @@ fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float*
 
 fd_status col_sqnorms(fd_ctx* c, const float* A, int64_t lda, int p, int64_t N, double* out_dev) {
     if (p < 1) return FD_OK;
+    if (N < 1) {
+        FD_CUDA(c, cudaMemsetAsync(out_dev, 0, (size_t)p * sizeof(double), c->stream));
+        return FD_OK;
+    }
     k_col_sqnorms<<<(unsigned)p, 1024, 0, c->stream>>>(A, lda, N, out_dev);
     FD_LAUNCH_CHECK(c, "k_col_sqnorms");
     return FD_OK;
@@ -236,20 +244,22 @@ fd_status scale_cols(fd_ctx* c, float* A, int64_t lda, int p, const float* f_dev
     return FD_OK;
 }
 
-fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, uint32_t seed) {
-    k_random_fill<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(A, lda, p, N, seed);
+fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, int64_t row0, uint32_t seed) {
+    if (N < 1 || p < 1) return FD_OK;
+    k_random_fill<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(A, lda, p, N, row0, seed);
     FD_LAUNCH_CHECK(c, "k_random_fill");
     return FD_OK;
 }
 
 fd_status sqrt_vec(fd_ctx* c, const float* d, float* out, int64_t N) {
+    if (N < 1) return FD_OK;
     k_sqrt_vec<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(d, out, N);
     FD_LAUNCH_CHECK(c, "k_sqrt_vec");
     return FD_OK;
 }
 
 fd_status copy_cols(fd_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd, int p, int64_t N) {
-    if (p < 1) return FD_OK;
+    if (p < 1 || N < 1) return FD_OK;
     FD_CUDA(c, cudaMemcpy2DAsync(dst, (size_t)ldd * 4, src, (size_t)lds * 4, (size_t)N * 4, (size_t)p,
                                  cudaMemcpyDeviceToDevice, c->stream));
     return FD_OK;

@@ -17,7 +17,9 @@ fd_status nn_product(fd_ctx* c, const float* A, int64_t lda, int m, const float*
 fd_status col_sqnorms(fd_ctx* c, const float* A, int64_t lda, int p, int64_t N, double* out_dev);
 fd_status d2f(fd_ctx* c, const double* in, float* out, int64_t n, double scale);
 fd_status scale_cols(fd_ctx* c, float* A, int64_t lda, int p, const float* f_dev, int64_t N);
-fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, uint32_t seed);
+// Counter-based uniform(-1, 1) fill of N rows x p columns; row i of A is row row0 + i of the stream, so a row range of
+// a larger block gets the values the whole block would.
+fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, int64_t row0, uint32_t seed);
 fd_status sqrt_vec(fd_ctx* c, const float* d, float* out, int64_t N);
 fd_status copy_cols(fd_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd, int p, int64_t N);
 

@@ -14,6 +14,11 @@
 // Vectors are fp32; every inner product and the small eigenproblem are fp64, and the measured
 // Gram matrix Q^T Q corrects the projected problem to first order, so fp32 loss of
 // orthogonality does not reach the Ritz values.
+//
+// Row-sharded contexts: every rank keeps rows [r0, r0 + n) of Q, W and the work blocks (pitch N, same addresses as
+// the unsharded layout), all tall-skinny products run on those rows, every reduced quantity that reaches the host
+// is summed over the ranks there (so all ranks take the same decisions), and the rows of a new block are gathered
+// from their owners before M is applied to it.
 #include <algorithm>
 #include <chrono>
 #include <cmath>
@@ -32,7 +37,8 @@ inline double secs(clk::time_point a, clk::time_point b) { return std::chrono::d
 
 struct Solver {
     fd_ctx* c;
-    int64_t N;
+    int64_t N;                      // pitch of every tall matrix = number of points
+    int64_t r0, n;                  // rows this rank owns (0, N unless the context is row-sharded)
     int m_cap, BP;
     float *Q, *W, *X;               // N x m_cap each (X = spare for out-of-place updates)
     float *R, *R2;                  // N x BP each
@@ -46,10 +52,10 @@ struct Solver {
     int applies = 0, restarts = 0;
     double t_apply = 0.0;
 
-    fd_status to_host(int n) {
-        FD_CUDA(c, cudaMemcpyAsync(h_out.data(), d_out, sizeof(double) * (size_t)n, cudaMemcpyDeviceToHost, c->stream));
+    fd_status to_host(int cnt) {
+        FD_CUDA(c, cudaMemcpyAsync(h_out.data(), d_out, sizeof(double) * (size_t)cnt, cudaMemcpyDeviceToHost, c->stream));
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
-        return FD_OK;
+        return allreduce_host(c, h_out.data(), cnt);
     }
     // The staging ring lives in the context (pinned HOST memory, allocated once): an upload never waits for the stream
     // unless its slot is still in flight.
@@ -75,11 +81,13 @@ struct Solver {
     }
 
     // W[:, c0 : c0 + n) = M Q[:, c0 : c0 + n), in blocks of at most bw columns
-    fd_status apply_cols(int c0, int n, int bw) {
+    fd_status apply_cols(int c0, int cnt, int bw) {
         auto t0 = clk::now();
-        for (int o = 0; o < n; o += bw) {
-            int w = std::min(bw, n - o);
-            FD_TRY(fd_apply(c, Q + (int64_t)(c0 + o) * N, N, w, W + (int64_t)(c0 + o) * N, N, FD_PREC_FP32));
+        FD_TRY(gather_rows(c, Q + (int64_t)c0 * N, N, cnt));         // the product needs all rows of the right block
+        for (int o = 0; o < cnt; o += bw) {
+            int w = std::min(bw, cnt - o);
+            FD_TRY(apply_general(c, c->beta, c->s(), c->s(), false, nullptr, N, 0, Q + (int64_t)(c0 + o) * N, N, w,
+                                 W + (int64_t)(c0 + o) * N, N, FD_PREC_FP32, /*gather_out=*/false));
             ++applies;
         }
         FD_TRY(tc_check_status(c));
@@ -92,7 +100,7 @@ struct Solver {
         dst.assign((size_t)m1 * m2, 0.0);
         for (int c0 = 0; c0 < m2; c0 += BP) {
             int w = std::min(BP, m2 - c0);
-            FD_TRY(tn_product(c, A, N, m1, B + (int64_t)c0 * N, N, w, N, d_out, d_scr, scr_n));
+            FD_TRY(tn_product(c, A + r0, N, m1, B + (int64_t)c0 * N + r0, N, w, n, d_out, d_scr, scr_n));
             FD_TRY(to_host(m1 * w));
             std::copy(h_out.begin(), h_out.begin() + (size_t)m1 * w, dst.begin() + (size_t)c0 * m1);
         }
@@ -139,7 +147,7 @@ struct Solver {
     // (eigenvalue of the unit-diagonal Gram matrix below drop_tol) are dropped.  Result in B, p updated.
     fd_status orthonormalise(float*& B, float*& spare, int& p, double drop_tol) {
         if (p == 0) return FD_OK;
-        FD_TRY(tn_product(c, B, N, p, B, N, p, N, d_out, d_scr, scr_n));
+        FD_TRY(tn_product(c, B + r0, N, p, B + r0, N, p, n, d_out, d_scr, scr_n));
         FD_TRY(to_host(p * p));
         std::vector<double> g((size_t)p * p), dinv(p);
         for (int j = 0; j < p; ++j) {
@@ -163,7 +171,7 @@ struct Solver {
             for (int i = 0; i < p; ++i) S[i + (size_t)jj * p] = (float)(dinv[i] * U[i + (size_t)j * p] * f);
         }
         FD_TRY(upload_S(S));
-        FD_TRY(nn_product(c, B, N, p, d_S, p, pk, spare, N, 1.f, 0.f, N));
+        FD_TRY(nn_product(c, B + r0, N, p, d_S, p, pk, spare + r0, N, 1.f, 0.f, n));
         std::swap(B, spare);
         p = pk;
         return FD_OK;
@@ -172,9 +180,17 @@ struct Solver {
     // B <- B - Q[:, 0:mq) (Q^T B), once.
     fd_status project_out(float* B, int p, int mq) {
         if (p == 0 || mq == 0) return FD_OK;
-        FD_TRY(tn_product(c, Q, N, mq, B, N, p, N, d_out, d_scr, scr_n));
-        FD_TRY(d2f(c, d_out, d_S, (int64_t)mq * p, -1.0));
-        FD_TRY(nn_product(c, Q, N, mq, d_S, mq, p, B, N, 1.f, 1.f, N));
+        FD_TRY(tn_product(c, Q + r0, N, mq, B + r0, N, p, n, d_out, d_scr, scr_n));
+        if (c->sh.on) {
+            // the coefficients are sums over the ranks: through the host, like every other projection
+            FD_TRY(to_host(mq * p));
+            std::vector<float> S((size_t)mq * p);
+            for (size_t i = 0; i < S.size(); ++i) S[i] = (float)(-h_out[i]);
+            FD_TRY(upload_S(S));
+        } else {
+            FD_TRY(d2f(c, d_out, d_S, (int64_t)mq * p, -1.0));
+        }
+        FD_TRY(nn_product(c, Q + r0, N, mq, d_S, mq, p, B + r0, N, 1.f, 1.f, n));
         return FD_OK;
     }
 };
@@ -200,7 +216,8 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
     if (L.m_max < 2 * nwant + b && L.m_max < N) return fail(c, FD_ERR_WORKSPACE, "m_max = %d < 2 (k + 1) + b = %d", L.m_max, 2 * nwant + b);
 
     Solver S;
-    S.c = c; S.N = N; S.BP = L.BP;
+    S.c = c; S.N = N; S.r0 = c->row0(); S.n = c->rows(); S.BP = L.BP;
+    const int64_t r0 = S.r0, n = S.n;
     S.m_cap = (int)std::min<int64_t>(L.m_max, N);
     const int m_cap = S.m_cap;
     S.Q = c->at<float>(L.eig_q); S.W = c->at<float>(L.eig_w); S.X = c->at<float>(L.eig_x);
@@ -221,17 +238,17 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
     const int nsel_max = nwant + buffer;
 
     // ---- start basis: Perron vector, then the warm-start columns or a random block ----------
-    FD_TRY(sqrt_vec(c, c->d(), S.Q, N));
+    FD_TRY(sqrt_vec(c, c->d() + r0, S.Q + r0, n));
     int cols = 1;
     const int room = std::max(0, m_cap - b - 1);                 // leave space for one expansion block
     if (Q0_dev) {
         int take = std::min(q0_cols, std::max(room, std::min(m_cap - 1, nwant)));
         take = std::min(take, m_cap - 1);
-        FD_TRY(copy_cols(c, Q0_dev, ldq0, S.Q + N, N, take, N));
+        FD_TRY(copy_cols(c, Q0_dev + r0, ldq0, S.Q + N + r0, N, take, n));
         cols += take;
     } else {
         int take = std::min(std::max(b, 1), m_cap - 1);
-        if (take > 0) FD_TRY(random_fill(c, S.Q + N, N, take, N, 0x5EEDu));
+        if (take > 0) FD_TRY(random_fill(c, S.Q + N + r0, N, take, n, r0, 0x5EEDu));
         cols += take;
     }
     {
@@ -313,9 +330,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
                     }
                 }
                 FD_TRY(S.upload_S(Sx));
-                FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
-                FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
-                FD_TRY(col_sqnorms(c, S.R, N, w, N, S.d_out));
+                FD_TRY(nn_product(c, S.W + r0, N, m, S.d_S, m, w, S.R + r0, N, 1.f, 0.f, n));
+                FD_TRY(nn_product(c, S.Q + r0, N, m, S.d_S + (size_t)m * w, m, w, S.R + r0, N, 1.f, 1.f, n));
+                FD_TRY(col_sqnorms(c, S.R + r0, N, w, n, S.d_out));
                 FD_TRY(S.to_host(w));
                 for (int jj = 0; jj < w; ++jj) resid[act[a0 + jj]] = std::sqrt(std::max(0.0, S.h_out[jj]));
             }
@@ -377,12 +394,12 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
                     Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[pick[jj]] * Xr[i + (size_t)pick[jj] * m]);
                 }
             FD_TRY(S.upload_S(Sx));
-            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
-            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+            FD_TRY(nn_product(c, S.W + r0, N, m, S.d_S, m, w, S.R + r0, N, 1.f, 0.f, n));
+            FD_TRY(nn_product(c, S.Q + r0, N, m, S.d_S + (size_t)m * w, m, w, S.R + r0, N, 1.f, 1.f, n));
             FD_TRY(S.upload_S(Sk));
-            FD_TRY(nn_product(c, S.Q, N, m, S.d_S, m, keep, S.X, N, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.Q + r0, N, m, S.d_S, m, keep, S.X + r0, N, 1.f, 0.f, n));
             std::swap(S.Q, S.X);                                  // X now holds the old basis: reuse it for W
-            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, keep, S.X, N, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.W + r0, N, m, S.d_S, m, keep, S.X + r0, N, 1.f, 0.f, n));
             std::swap(S.W, S.X);
             S.m = keep;
             ++S.restarts;
@@ -396,8 +413,8 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
                     Sx[(size_t)m * w + i + (size_t)jj * m] = (float)(-theta[pick[jj]] * Xr[i + (size_t)pick[jj] * m]);
                 }
             FD_TRY(S.upload_S(Sx));
-            FD_TRY(nn_product(c, S.W, N, m, S.d_S, m, w, S.R, N, 1.f, 0.f, N));
-            FD_TRY(nn_product(c, S.Q, N, m, S.d_S + (size_t)m * w, m, w, S.R, N, 1.f, 1.f, N));
+            FD_TRY(nn_product(c, S.W + r0, N, m, S.d_S, m, w, S.R + r0, N, 1.f, 0.f, n));
+            FD_TRY(nn_product(c, S.Q + r0, N, m, S.d_S + (size_t)m * w, m, w, S.R + r0, N, 1.f, 1.f, n));
         }
         auto tp4 = clk::now();
         t_restart += secs(tp3, tp4);
@@ -412,7 +429,7 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             // the residuals lie (numerically) inside the basis: try a random direction, give up after a few
             if (++stagnation > 3) break;
             p = std::min<int64_t>(b, N - S.m);
-            FD_TRY(random_fill(c, S.R, N, p, N, 0xABCD1234u + (uint32_t)iter));
+            FD_TRY(random_fill(c, S.R + r0, N, p, n, r0, 0xABCD1234u + (uint32_t)iter));
             FD_TRY(S.project_out(S.R, p, S.m));
             FD_TRY(S.project_out(S.R, p, S.m));
             FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-5));
@@ -420,7 +437,7 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             FD_TRY(S.orthonormalise(S.R, S.R2, p, 1e-3));
             if (p == 0) break;
         }
-        FD_TRY(copy_cols(c, S.R, N, S.Q + (int64_t)S.m * N, N, p, N));
+        FD_TRY(copy_cols(c, S.R + r0, N, S.Q + (int64_t)S.m * N + r0, N, p, n));
         auto tp5 = clk::now();
         t_orth += secs(tp4, tp5);
         FD_TRY(S.apply_cols(S.m, p, b));
@@ -439,8 +456,9 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
             for (int jj = 0; jj < w; ++jj)
                 for (int i = 0; i < m; ++i) Sx[i + (size_t)jj * m] = (float)Xr[i + (size_t)(c0 + jj) * m];
             FD_TRY(S.upload_S(Sx));
-            FD_TRY(nn_product(c, S.Q, N, m, S.d_S, m, w, evecs_dev + (int64_t)c0 * ldv, ldv, 1.f, 0.f, N));
+            FD_TRY(nn_product(c, S.Q + r0, N, m, S.d_S, m, w, evecs_dev + (int64_t)c0 * ldv + r0, ldv, 1.f, 0.f, n));
         }
+        FD_TRY(gather_rows(c, evecs_dev, ldv, nout));              // complete eigenvectors on every rank
         for (int i = 0; i < nwant; ++i) evals_host[i] = i < nout ? theta[i] : 0.0;
         FD_CUDA(c, cudaStreamSynchronize(c->stream));
     }

@@ -65,6 +65,14 @@ struct fd_ctx {
     float* stage[kStageSlots] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t stage_ev[kStageSlots] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_floats = 0;
+    // row-sharded operation (fd_set_shard): this rank owns rows [r0, r1) of every quadratic pass
+    struct Shard {
+        bool on = false;
+        fd_shard h{};                // callbacks, rank, world, exchange buffer
+        int64_t chunk = 0, r0 = 0, r1 = 0;
+    } sh;
+    int64_t row0() const { return sh.on ? sh.r0 : 0; }
+    int64_t rows() const { return sh.on ? sh.r1 - sh.r0 : L.N; }
 
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
     float* xs() const { return at<float>(L.xs); }
@@ -126,7 +134,16 @@ fd_status apply_dispatch(fd_ctx* c, const ApplyArgs& a);
 // row-sum (V == nullptr) with a right vector take the same kernel family as the block products of the same operator.
 fd_status apply_general(fd_ctx* c, double beta, const float* left_dev, const float* right_dev, bool right_pos,
                         const float* Xrow_dev, int64_t Nrow, int64_t ldxrow, const float* V_dev, int64_t ldv, int32_t b,
-                        float* Y_dev, int64_t ldy, fd_precision prec);
+                        float* Y_dev, int64_t ldy, fd_precision prec, bool gather_out = true);
+
+// ---- row-sharded operation (fd_shard.cu) ----------------------------------------------------------
+// Rows [begin, end) of rank `rank`: contiguous ranges of round_up(ceil(N / world), 256) rows.
+void shard_range(int64_t N, int world, int rank, int64_t* begin, int64_t* end);
+// A is column-major with pitch lda and `cols` columns; on entry every rank holds valid values in its own rows, on
+// return in all N rows.  No-op for an unsharded context.  cols is split into groups of at most b_max internally.
+fd_status gather_rows(fd_ctx* c, float* A, int64_t lda, int cols);
+// In-place sum over the ranks of n host doubles.  No-op for an unsharded context.
+fd_status allreduce_host(fd_ctx* c, double* buf, int64_t n);
 // Reads and clears the tensor-core kernel's status word; FD_ERR_TIMEOUT if a bounded wait expired.  Synchronises.
 fd_status tc_check_status(fd_ctx* c);
 // Launches a one-thread kernel whose bounded wait must expire after limit_cycles (test of the time-out plumbing).
