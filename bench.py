@@ -12,7 +12,10 @@ time to k eigenpairs on the five benchmark configurations.
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--n LOG2N]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU float64 oracle on a bounded row sample of the same
-workload instead.  `--gpus N` without a launcher starts N ranks itself (one per GPU, independent replicas).
+workload instead.  `--gpus N` without a launcher starts N ranks itself, one per GPU.  With N > 1 the data set is row-
+sharded (Sec. 3 of the paper): every rank holds all points and evaluates N / world rows of every quadratic pass, the
+rows of each result are gathered over NCCL, so the total work is fixed ("scaling": "strong") and `value` is the one
+job's N^2 b over the slowest rank's time.  `--replicas` runs N independent copies instead ("weak").
 """
 from __future__ import annotations
 
@@ -175,7 +178,8 @@ def max_over_ranks(values, dist, device):
 
 
 def job_value(units_per_rank: float, world: int, ms: float) -> float:
-    """Whole-job throughput of `world` independent replicas (weak scaling): all units over the slowest rank's time."""
+    """Whole-job throughput: the units all ranks processed over the slowest rank's time.  Independent replicas process
+    the full workload each; row-sharded ranks process 1 / world of one workload each."""
     return units_per_rank * world / (ms * 1e-3)
 
 
@@ -203,14 +207,25 @@ def run_gpu(args):
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     dist = None
-    if world > 1:
+    if world > 1 or args.force_shard:
         import torch.distributed as dist_mod
         dist = dist_mod
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if world == 1:                       # --force-shard on one GPU: a one-rank NCCL group exercises the exchange path
+            os.environ.setdefault("MASTER_PORT", str(free_port()))
+            os.environ.setdefault("RANK", "0")
+            os.environ.setdefault("WORLD_SIZE", "1")
         torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        import datetime
+        # generous: in replica mode the other ranks wait at the last barrier while rank 0 runs the eigensolver leg
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local), timeout=datetime.timedelta(minutes=60))
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    sharded = dist is not None and not args.replicas
+    transport = None
+    if sharded:
+        # rows gathered on the NCCL group, the eigensolver's small host sums on a gloo group
+        transport = fd.TorchDistTransport(rank, world, group=None, host_group=dist.new_group(backend="gloo"))
 
     X, V, cfg = workload(args.n)
     N, b, beta, alpha = cfg["N"], cfg["b"], cfg["beta"], cfg["alpha"]
@@ -224,6 +239,11 @@ def run_gpu(args):
     if args.path:
         ctx.set_option("path", {"auto": 0, "simt": 1, "tc": 2}[args.path])
     stream = torch.cuda.current_stream(dev)
+    shard = fd.Shard(transport, N, b, dev, stream=stream) if sharded else None
+    if sharded:
+        ctx.set_shard(shard)
+    cfg["parallelism"] = (f"rows sharded over {world} ranks, result rows gathered (NCCL all-gather)" if sharded else
+                          f"{world} independent replicas" if world > 1 else "single GPU")
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -306,6 +326,8 @@ def run_gpu(args):
         c2 = fd.Context(Xd, b_max=b, m_max=0)
         if args.path:
             c2.set_option("path", {"auto": 0, "simt": 1, "tc": 2}[args.path])
+        if sharded:
+            c2.set_shard(shard)
         c2.degree(beta, alpha)
         c2.apply(Vd, out=Yd)
         Yh.copy_(Yd.t(), non_blocking=True)
@@ -325,14 +347,15 @@ def run_gpu(args):
 
     total_ms, e2e_ms, deg_ms, app_ms = max_over_ranks([total_ms, e2e_ms, deg_ms, app_ms], dist, dev)
     step_ms = total_ms / args.steps
-    units = float(N) * N * b                      # pair-columns of one block product
+    # pair-columns one rank processes per block product: all of them as a replica, its rows' share when sharded
+    units = float(N) * N * b / (world if sharded else 1)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         rates = fd.fd_unit_peaks(dev)
         D = cfg["D"]
         sm_max = float(peaks.get("sm_max_mhz", 1965.0))
-        pairs_per_s = float(N) * N / (app_ms * 1e-3)
+        pairs_per_s = units / b / (app_ms * 1e-3)                 # per GPU: the roofline is one GPU's
         mufu_peak = rates["sm_count"] * rates["ex2_per_clk_sm"] * sm_max * 1e6         # exp / s at the maximum SM clock
         fma_peak = rates["sm_count"] * rates["ffma_per_clk_sm"] * sm_max * 1e6
         if path_used == "simt":
@@ -357,40 +380,44 @@ def run_gpu(args):
                                                  "product_24_mma_ts_n64": 24 * rates["clk_mma_ts_n64"],
                                                  "mufu_128x128_exps": 128 * 128 / rates["ex2_per_clk_sm"]},
                     "unit_rates": rates}
-        deg_pairs_per_s = 2.0 * float(N) * N / (deg_ms * 1e-3)
+        deg_pairs_per_s = 2.0 * units / b / (deg_ms * 1e-3)       # per GPU
         out = {"metric": METRIC, "value": job_value(units, world, app_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-               "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+               "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
                "apply_ms": app_ms, "path": path_used, "roofline": roofline,
-               "whole_step": {"ms": step_ms, "pair_cols_per_s": job_value(float(N) * N * (b + 2), world, step_ms),
+               "whole_step": {"ms": step_ms, "pair_cols_per_s": job_value(units * (b + 2) / b, world, step_ms),
                               "note": "degree pass + second normalisation pass + scale vector + block product"},
                "degree_passes": {"ms_both": deg_ms, "pairs_per_s": deg_pairs_per_s, "frac_of_mufu_peak": deg_pairs_per_s / mufu_peak},
                "fast_mode_apply": None if fast_ms is None else {
-                   "ms": fast_ms, "pair_cols_per_s": units / (fast_ms * 1e-3), "frac_of_mufu_peak": float(N) * N / (fast_ms * 1e-3) / mufu_peak,
+                   "ms": fast_ms, "pair_cols_per_s": units / (fast_ms * 1e-3), "frac_of_mufu_peak": units / b / (fast_ms * 1e-3) / mufu_peak,
                    "note": "FD_PREC_FAST: single fp16 operands, relative Frobenius error ~2e-4 (bound 3e-3); reported separately"},
                "e2e": {"value": job_value(units, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                        "note": "host buffers: H2D of X and V, fd_create, degree passes, block product, D2H of Y",
                        "h2d_bytes_per_step": int(Xh.numel() * 4 + Vh.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 4)},
                "gpu_launches": int(launches), "workspace_bytes": ctx.workspace_bytes}
-        if not args.no_cpu:
+        if not args.no_cpu and world == 1:
             out["cpu_baseline"] = cpu_baseline(X, V, cfg)
-        ctx.close()
-        if not args.no_eigs:
-            del Xd, Vd, Yd
-            torch.cuda.empty_cache()
-            out["time_to_k_eigs"] = time_to_k_eigs(fd, dev, args)
-        print(json.dumps(out), flush=True)
     ctx.close()
+    if not args.no_eigs and (rank == 0 or sharded):
+        # one GPU or replicas: rank 0 alone; row-sharded: every rank takes part in the sharded solves
+        del Xd, Vd, Yd
+        torch.cuda.empty_cache()
+        eigs = time_to_k_eigs(fd, dev, args, transport if sharded else None)
+        if rank == 0:
+            out["time_to_k_eigs"] = eigs
+    if rank == 0:
+        print(json.dumps(out), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
 
 
-def time_to_k_eigs(fd, dev, args):
+def time_to_k_eigs(fd, dev, args, transport=None):
     """Second half of the metric: wall time from a fresh bandwidth to k eigenpairs (degree passes + fd_eigs) on the five
     benchmark configurations at their full sizes (C2 at all four bandwidths; non-convergence within the apply budget is a
     reported outcome there), the whole dyadic bandwidth flow on C3, and the nested-level ladder with the bandwidth
-    re-optimised on every level.  Host wall clock around synchronous calls."""
+    re-optimised on every level.  Host wall clock around synchronous calls.  With a transport (row-sharded ranks) every
+    rank runs the same solves on its rows; only the large configurations are run then (C3 with its flow, C4, C5)."""
     import torch
     import workloads
     res = []
@@ -404,6 +431,8 @@ def time_to_k_eigs(fd, dev, args):
              ("C4 latent torus R^30", workloads.latent_torus(262144, seed=42), 32, 32, 2.0, 600)]
     if not args.no_c5_eigs:
         cases.append(("C5 6-torus", workloads.torus6(1 << 20, seed=42), 128, 64, 2.0, 400))
+    if transport is not None:
+        cases = [cse for cse in cases if cse[0][:2] in ("C3", "C4", "C5")]
     if args.eigs_case:
         # restrict the leg to one configuration (for profiling a single solve); C2 keeps its four bandwidths
         pts = None
@@ -421,6 +450,8 @@ def time_to_k_eigs(fd, dev, args):
         X = torch.from_numpy(Xnp).to(dev)
         m_max = default_m_max(k, b)
         ctx = fd.Context(X, b_max=b, m_max=m_max)
+        if transport is not None:
+            ctx.set_shard(fd.Shard(transport, N, b, dev))
         ctx.degree(beta, 1.0)                                        # warm-up of both passes
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
@@ -445,7 +476,7 @@ def time_to_k_eigs(fd, dev, args):
         del ctx, X
         torch.cuda.empty_cache()
         res.append(rec)
-    if not args.eigs_case:
+    if not args.eigs_case and transport is None:
         res.append(ladder(fd, dev, args.ladder_full))
     return res
 
@@ -525,6 +556,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n", type=int, default=20, help="log2 of the number of points (default 20: the headline size)")
     ap.add_argument("--path", default="", choices=["", "auto", "simt", "tc"])
+    ap.add_argument("--replicas", action="store_true", help="with --gpus N > 1: N independent replicas instead of row sharding")
+    ap.add_argument("--force-shard", action="store_true", help="one GPU: run the row-sharded code path on a one-rank NCCL group")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--no-eigs", action="store_true", help="skip the time-to-k-eigenpairs leg")
     ap.add_argument("--no-c5-eigs", action="store_true", help="skip the eigensolve at N = 2^20 (k = 128, b = 64; about 80 s)")
