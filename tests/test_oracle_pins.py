@@ -390,3 +390,46 @@ def test_principal_angles_two_distinct_angles_and_nonorthonormal_columns():
     assert dense.principal_angles(A, A @ Ta).max() < 1e-12
     C = np.zeros((n, 2)); C[4, 0] = 1.0; C[5, 1] = 1.0
     assert np.allclose(dense.principal_angles(A, C), [np.pi / 2, np.pi / 2])
+
+
+# ------------------------------------------------------------------ the T^6 validation score (Sec. 3, Fig. 1(c))
+def test_rv_overlap_closed_forms():
+    from oracle import overlap
+    rng = np.random.default_rng(3)
+    n = 4000
+    # three exactly orthonormal, exactly centred directions (discrete Fourier modes on n points)
+    t = 2.0 * np.pi * np.arange(n) / n
+    c1, s1, c2, s2 = np.cos(t), np.sin(t), np.cos(2 * t), np.sin(2 * t)
+    B = np.stack([c1, s1], axis=1)
+    # identical span, any basis of it, any offset: 1
+    T = np.array([[2.0, -0.7], [0.4, 1.3]])
+    assert overlap.rv_overlap(B @ T + 5.0, B) == pytest.approx(1.0, abs=1e-12)
+    # orthogonal span: 0
+    assert overlap.rv_overlap(np.stack([c2, s2], axis=1), B) == pytest.approx(0.0, abs=1e-12)
+    # one shared direction of two: 1/2
+    assert overlap.rv_overlap(np.stack([c1, c2], axis=1), B) == pytest.approx(0.5, abs=1e-12)
+    # both directions tilted by known angles out of the span: (cos^2 a + cos^2 b) / 2
+    a, b = 0.3, 1.1
+    A = np.stack([np.cos(a) * c1 + np.sin(a) * c2, np.cos(b) * s1 + np.sin(b) * s2], axis=1)
+    assert overlap.rv_overlap(A, B) == pytest.approx((np.cos(a) ** 2 + np.cos(b) ** 2) / 2.0, abs=1e-12)
+    # symmetric in its arguments; invariant under a rotation inside the doublet (the degenerate pair may rotate)
+    R = np.array([[np.cos(0.9), -np.sin(0.9)], [np.sin(0.9), np.cos(0.9)]])
+    assert overlap.rv_overlap(B, A) == pytest.approx(overlap.rv_overlap(A, B @ R), abs=1e-12)
+    # random data: strictly between 0 and 1
+    v = overlap.rv_overlap(rng.standard_normal((n, 2)), B)
+    assert 0.0 <= v < 0.01
+    assert np.allclose(overlap.first_harmonic_target(np.stack([t] * 6, axis=1), 5), B)
+
+
+def test_t6_first_harmonic_overlap_soft_pin(golden_dir):
+    # Paper's T^6 run at N = 1024: printed overlap 0.929 (another RNG): the oracle flow's leading doublet must score in the
+    # same range (1 - overlap within a factor of three of the printed 0.071) against the largest circle, and far lower
+    # against any other circle
+    from oracle import overlap
+    X, ang = workloads.torus6_paper(1024, seed=42, return_angles=True)
+    bx, status, log = flow.beta_flow(flow.dense_probe(X, 0.5, 3), 1024, flow.beta0(X), 1000.0)
+    lam, U, d = dense.eigs(X, bx, 0.5, 3)
+    psi = dense.markov_vectors(U, d)
+    score = overlap.rv_overlap(psi[:, 1:3], overlap.first_harmonic_target(ang, 5))
+    assert 0.071 / 3.0 < 1.0 - score < 0.071 * 3.0
+    assert overlap.rv_overlap(psi[:, 1:3], overlap.first_harmonic_target(ang, 0)) < 0.2

@@ -54,7 +54,7 @@ def torus_grid(N1: int, N2: int) -> np.ndarray:
 
 
 def torus6(N: int = 131072, seed: int = 42, sigma: float = 0.01,
-           radii=(1.0,) * 6, pad_to: int | None = None) -> np.ndarray:
+           radii=(1.0,) * 6, pad_to: int | None = None, return_angles: bool = False):
     """Draw order: t = uniform(0, 2 pi, (N, 6)); noise = standard_normal((N, 12)).
 
     x = (R_a cos t_a, R_a sin t_a)_{a=1..6} + sigma * noise.  The level-n subsample
@@ -70,12 +70,15 @@ def torus6(N: int = 131072, seed: int = 42, sigma: float = 0.01,
         x += sigma * rng.standard_normal((N, 12))
     if pad_to is not None and pad_to > 12:
         x = np.concatenate([x, np.zeros((N, pad_to - 12))], axis=1)
+    if return_angles:
+        return x.astype(np.float32), t
     return x.astype(np.float32)
 
 
-def torus6_paper(N: int, seed: int = 42) -> np.ndarray:
-    """The paper's Sec. 3 / App. B shape: anisotropic radii, no noise, D = 32 (12 non-zero)."""
-    return torus6(N, seed=seed, sigma=0.0, radii=PAPER_T6_RADII, pad_to=32)
+def torus6_paper(N: int, seed: int = 42, return_angles: bool = False):
+    """The paper's Sec. 3 / App. B shape: anisotropic radii, no noise, D = 32 (12 non-zero).  With return_angles the
+    N x 6 angles come back too (they enter only the post-hoc first-harmonic score, never a solve)."""
+    return torus6(N, seed=seed, sigma=0.0, radii=PAPER_T6_RADII, pad_to=32, return_angles=return_angles)
 
 
 _VM_MEANS = np.array([(-1.4, 2.6), (-1.4, -0.7), (1.1, -0.8), (-2.5, 2.9)], dtype=np.float64)
