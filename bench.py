@@ -478,7 +478,54 @@ def time_to_k_eigs(fd, dev, args, transport=None):
         res.append(rec)
     if not args.eigs_case and transport is None:
         res.append(ladder(fd, dev, args.ladder_full))
+        res.append({"t6_validation": t6_validation(fd, dev, args.t6_full)})
     return res
+
+
+def t6_validation(fd, dev, full=False):
+    """The paper's T^6 validation sweep (Sec. 3, Fig. 1(b), 1(c)): anisotropic radii, alpha = 1/2, k = 3, seed 42 per N, the
+    bandwidth flow from beta_0 of Eq. 7; per N the selected beta_x and the post-hoc squared-RV overlap of the leading two
+    nontrivial Markov modes with (cos, sin) of the largest circle, with the printed values beside them (another RNG).
+    Default N = 2^10 ... 2^17; --t6-full continues to 2^20."""
+    import torch
+    import workloads
+    printed = {}
+    try:
+        with open(os.path.join(ROOT, "tests", "golden", "t6_bandwidth_table.txt")) as f:
+            for line in f:
+                if line[0].isdigit():
+                    r = line.strip().split(",")
+                    printed[int(r[0])] = (float(r[1]), float(r[3]))
+    except OSError:
+        pass
+    out = []
+    for e in range(10, 21 if full else 18):
+        N = 1 << e
+        X, ang = workloads.torus6_paper(N, seed=42, return_angles=True)
+        ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        bx, outcome, lam, U, recs = ctx.beta_flow(3, 8, 0.5, beta_start=0.0, beta_max=1000.0)
+        dt = time.perf_counter() - t0
+        psi = ctx.scale_by_degree(U, -0.5).cpu().numpy().astype(np.float64)[:, 1:3]
+        path = "tc" if ctx.get_option("last_path") == 2 else "simt"
+        ctx.close()
+        # squared RV coefficient of the two centred 2-column blocks (float64, whitened cross-covariance)
+        A = psi - psi.mean(axis=0)
+        B = np.stack([np.cos(ang[:, 5]), np.sin(ang[:, 5])], axis=1)
+        B = B - B.mean(axis=0)
+
+        def inv_sqrt(G):
+            w, Q = np.linalg.eigh(G)
+            return (Q / np.sqrt(w)) @ Q.T
+        C = inv_sqrt(A.T @ A) @ (A.T @ B) @ inv_sqrt(B.T @ B)
+        score = float((C * C).sum() / 2.0)
+        rec = {"N": N, "beta_x": bx, "outcome": outcome, "probes": len(recs), "applies": int(sum(r["applies"] for r in recs)),
+               "flow_s": dt, "path": path, "n_eff": recs[-1]["n_eff"], "d_hat": recs[-1]["d_hat"], "one_minus_overlap": 1.0 - score}
+        if N in printed:
+            rec["printed_beta_x"], rec["printed_one_minus_overlap"] = printed[N][0], 1.0 - printed[N][1]
+        out.append(rec)
+    return out
 
 
 def default_m_max(k, b):
@@ -563,6 +610,7 @@ def main():
     ap.add_argument("--no-c5-eigs", action="store_true", help="skip the eigensolve at N = 2^20 (k = 128, b = 64; about 80 s)")
     ap.add_argument("--eigs-case", default="", choices=["", "C1", "C2", "C3", "C4", "C5"],
                     help="time-to-k-eigenpairs leg: only this configuration (and no ladder)")
+    ap.add_argument("--t6-full", action="store_true", help="T^6 validation sweep up to N = 2^20 instead of 2^17")
     ap.add_argument("--ladder-full", action="store_true", help="run config 5's own ladder (2^16 ... 2^20, k = 128, b = 64; many minutes)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
