@@ -129,3 +129,24 @@ def beta_flow(probe, N, beta_start, beta_max, eta=ETA["fp32"], ratio=2.0):
             return bv, "VERTEX", log
         beta *= ratio
     return log[-1]["beta"], "RIGHT_EDGE", log
+
+
+def cascade(probes, N, beta_start, beta_max, etas, ratio=2.0):
+    """Precision cascade (Sec. 2.3, last paragraph; eta per data type from the footnote to Eq. 11).
+
+    One sweep per requested data type, in the order given: `probes[s]` evaluates a probe at stage s (its arithmetic)
+    and `etas[s]` is that data type's precision scale in Eqs. 11-12.  The paper says only that the selected state of
+    one stage initialises the next; the reading taken here: stage s + 1 restarts the dyadic sweep one grid step below
+    the bandwidth stage s selected (so that a bracket around it can form) and the final bandwidth and eigenpairs
+    are those of the last stage.  Returns (beta_x, status, [log per stage]).
+    """
+    logs = []
+    start = float(beta_start)
+    bx, status = float("nan"), "PERRON_WALL"
+    for probe, eta in zip(probes, etas):
+        bx, status, log = beta_flow(probe, N, start, beta_max, eta=eta, ratio=ratio)
+        logs.append(log)
+        if not (bx == bx):                       # no safe probe at all in this stage: nothing to hand on
+            break
+        start = bx / ratio
+    return bx, status, logs

@@ -433,3 +433,37 @@ def test_t6_first_harmonic_overlap_soft_pin(golden_dir):
     score = overlap.rv_overlap(psi[:, 1:3], overlap.first_harmonic_target(ang, 5))
     assert 0.071 / 3.0 < 1.0 - score < 0.071 * 3.0
     assert overlap.rv_overlap(psi[:, 1:3], overlap.first_harmonic_target(ang, 0)) < 0.2
+
+
+def test_precision_cascade_by_hand():
+    # V_bias = 1 / beta, V_stat as in the bracket test (minimum of V_bias + V_stat near beta = 3), and a Perron gap
+    # g_P = 0.05 / beta that the coarse data type (eta = 1e-3: wall at g_P <= 1e-2, Eq. 12) loses at beta = 8 while fp32
+    # (eta = 1e-7) never does.  Stage 1 from beta = 0.25: its V_mach = (10 eta / g_P)^6 = (beta / 5)^6 moves the
+    # minimum to smaller beta; stage 2 must restart one grid step below stage 1's selection and find the fp32 vertex.
+    so = lambda b: 1e6 * b ** -3.0
+
+    def probe(beta):
+        return np.array([1.0, 1.0 - 0.05 / beta, math.exp(-1.0 / beta) * (1.0 - 0.05 / beta)]), so(beta), so(2 * beta)
+    # single-stage runs with each eta
+    bx_c, st_c, log_c = flow.beta_flow(probe, 1000, 0.25, 1000.0, eta=1e-3)
+    bx_f, st_f, log_f = flow.beta_flow(probe, 1000, 0.25, 1000.0, eta=1e-7)
+    assert st_c == "VERTEX" and st_f == "VERTEX" and bx_c < bx_f
+    bx, status, logs = flow.cascade([probe, probe], 1000, 0.25, 1000.0, [1e-3, 1e-7])
+    assert len(logs) == 2 and status == "VERTEX"
+    assert [r["beta"] for r in logs[0]] == [r["beta"] for r in log_c]                 # stage 1 = the coarse sweep
+    assert logs[1][0]["beta"] == bx_c / 2.0                                           # stage 2 restarts one step below it
+    assert [r["beta"] for r in logs[1][1:-1]] == [bx_c / 2.0 * 2 ** j for j in range(1, len(logs[1]) - 1)]
+    # same potential, same fp32 minimum: the cascade's final vertex agrees with the fp32-only sweep's to the accuracy of
+    # the three-point fit (different grid offsets)
+    assert abs(math.log(bx / bx_f)) < 0.1
+    assert all(r["V_mach"] < 1e-20 for r in logs[1])
+    # a first stage that meets the wall hands on its last safe probe
+    def probe_w(beta):
+        return np.array([1.0, 1.0 - min(0.9, 0.05 / beta ** 3), math.exp(-1.0 / beta) * 0.09]), so(beta), so(2 * beta)
+    bx1, st1, log1 = flow.beta_flow(probe_w, 1000, 0.25, 1000.0, eta=1e-3)
+    assert st1 == "PERRON_WALL" and bx1 == 1.0 and log1[-1]["beta"] == 2.0           # 0.05 / 8 = 6.25e-3 <= 1e-2
+    bx2, st2, logs2 = flow.cascade([probe_w, probe_w], 1000, 0.25, 1000.0, [1e-3, 1e-7])
+    assert logs2[1][0]["beta"] == 0.5 and st2 == "VERTEX" and bx2 > 2.0
+    # one stage = the plain flow
+    bx3, st3, logs3 = flow.cascade([probe], 1000, 0.25, 1000.0, [1e-7])
+    assert (bx3, st3) == (bx_f, st_f)
