@@ -472,6 +472,15 @@ def time_to_k_eigs(fd, dev, args, transport=None):
                            "beta_x": bx, "outcome": outcome, "probes": len(recs),
                            "applies": int(sum(r["applies"] for r in recs)), "n_eff_at_beta_x": recs[-1]["n_eff"],
                            "d_hat_at_beta_x": recs[-1]["d_hat"]}
+            # the same sweep as a precision cascade (Sec. 2.3): reduced-precision kernels explore, fp32-grade kernels resolve
+            t5 = time.perf_counter()
+            bxc, outc, lam3, U3, stg = ctx.beta_flow_cascade(k, b, 1.0, [(fd.FD_PREC_FAST, 0.0, 0.0), (fd.FD_PREC_FP32, 0.0, 0.0)],
+                                                             beta_start=1.0, beta_max=1000.0, max_applies=400)
+            t6 = time.perf_counter()
+            rec["cascade"] = {"stages": "FD_PREC_FAST (eta 1e-3, tol 1e-3) -> FD_PREC_FP32 (eta 1e-7, tol 1e-6)", "seconds": t6 - t5,
+                              "beta_x": bxc, "outcome": outc, "probes_per_stage": [len(x) for x in stg],
+                              "applies_per_stage": [int(sum(r["applies"] for r in x)) for x in stg],
+                              "max_eval_diff_vs_flow": float(abs(lam3 - lam2).max())}
         ctx.close()
         del ctx, X
         torch.cuda.empty_cache()

@@ -158,7 +158,7 @@ typedef struct {
     double lambda1;            /* first nontrivial eigenvalue                                 */
     int32_t applies;           /* block applies the probe's eigensolve took                   */
     int32_t flags;             /* bit 0: inadmissible (Eq. 12); bit 1: final (vertex) probe;  */
-                               /* bit 2: eigensolve stalled above tol (residuals <= 1e-4)     */
+                               /* bit 2: eigensolve stalled above tol (residuals <= max(1e-4, 100 tol)) */
 } fd_probe;
 
 typedef struct {
@@ -181,6 +181,27 @@ enum { FD_FLOW_VERTEX = 0, FD_FLOW_PERRON_WALL = 1, FD_FLOW_LEFT_EDGE = 2, FD_FL
 fd_status fd_beta_flow(fd_ctx* ctx, const fd_flow_opts* opts, const float* Q0_dev, int64_t ldq0,
                        int32_t q0_cols, fd_probe* log, int32_t* n_probes, int32_t* outcome,
                        double* beta_x_host, double* evals_host, float* evecs_dev, int64_t ldv);
+
+/* Precision cascade of Sec. 2.3 (last paragraph): one sweep per requested data type, in order; the state a stage
+ * selects initialises the next stage and the final bandwidth and eigenpairs are the last stage's.  Here a stage is a
+ * precision mode of the kernels (FD_PREC_FAST explores, FD_PREC_FP32 resolves) with its own precision scale eta in
+ * Eqs. 11-12 (footnote to Eq. 11: 8e-3 bf16, 1e-3 tf32, 1e-7 fp32; the reduced-precision mode here carries fp16
+ * operands and behaves like the tf32 entry) and its own eigensolver tolerance (a reduced-precision operator has a
+ * residual floor near its own error, about 2e-4).  Reading of "initialises": stage s + 1 restarts the dyadic sweep
+ * at beta_x(s) / ratio, warm-started from stage s's eigenvectors.  opts->eta and opts->tol are ignored (each stage
+ * has its own); everything else in opts applies to every stage.  log receives the probes of all stages back to
+ * back and stage_first_probe[s] (n_stages + 1 entries) the index of stage s's first record; outcome, beta_x, evals
+ * and evecs are the last stage's.  A stage that finds no admissible probe at all ends the cascade with
+ * FD_ERR_PERRON_WALL.  Synchronous. */
+typedef struct {
+    fd_precision prec;
+    double eta;                /* <= 0: 1e-7 for FD_PREC_FP32, 1e-3 for FD_PREC_FAST                        */
+    double tol;                /* <= 0: 1e-6 for FD_PREC_FP32, 1e-3 for FD_PREC_FAST                        */
+} fd_cascade_stage;
+fd_status fd_beta_flow_cascade(fd_ctx* ctx, const fd_flow_opts* opts, const fd_cascade_stage* stages, int32_t n_stages,
+                               const float* Q0_dev, int64_t ldq0, int32_t q0_cols, fd_probe* log, int32_t* n_probes,
+                               int32_t* stage_first_probe, int32_t* outcome, double* beta_x_host, double* evals_host,
+                               float* evecs_dev, int64_t ldv);
 
 /* Out-of-sample extension of Markov eigenvectors from the context's points to new points
  * (Sec. 1, the (n, beta) ladder): psi_j(x) = sum_i K(x, x_i) q_i^-alpha psi_j(x_i) /

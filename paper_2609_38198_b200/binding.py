@@ -25,7 +25,7 @@ FLOW_OUTCOMES = {0: "VERTEX", 1: "PERRON_WALL", 2: "LEFT_EDGE", 3: "RIGHT_EDGE"}
 # Every symbol include/fd.h declares (checked by the CPU test-suite against the header).
 EXPORTS = [
     "fd_workspace_bytes", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree",
-    "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_ladder_start", "fd_scale_by_degree",
+    "fd_apply", "fd_apply_general", "fd_synchronize", "fd_eigs", "fd_beta_flow", "fd_beta_flow_cascade", "fd_nystrom", "fd_ladder_start", "fd_scale_by_degree",
     "fd_apply_general_static", "fd_unit_peaks", "fd_shard_rows", "fd_shard_exchange_bytes", "fd_set_shard", "fd_status_string", "fd_last_error", "fd_version", "fd_launch_count",
 ]
 
@@ -52,6 +52,10 @@ class fd_flow_opts(Structure):
                 ("warm_start", c_int32)]
 
 
+class fd_cascade_stage(Structure):
+    _fields_ = [("prec", c_int32), ("eta", c_double), ("tol", c_double)]
+
+
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(f"{LIB_PATH} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
@@ -76,6 +80,9 @@ def _load() -> ctypes.CDLL:
     lib.fd_beta_flow.argtypes = [c_void_p, POINTER(fd_flow_opts), c_void_p, c_int64, c_int32, POINTER(fd_probe),
                                  POINTER(c_int32), POINTER(c_int32), POINTER(c_double), POINTER(c_double), c_void_p,
                                  c_int64]
+    lib.fd_beta_flow_cascade.argtypes = [c_void_p, POINTER(fd_flow_opts), POINTER(fd_cascade_stage), c_int32, c_void_p,
+                                         c_int64, c_int32, POINTER(fd_probe), POINTER(c_int32), POINTER(c_int32),
+                                         POINTER(c_int32), POINTER(c_double), POINTER(c_double), c_void_p, c_int64]
     lib.fd_nystrom.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int32, POINTER(c_double),
                                c_void_p, c_int64]
     lib.fd_ladder_start.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int32, POINTER(c_double),
@@ -83,7 +90,7 @@ def _load() -> ctypes.CDLL:
     lib.fd_ladder_start.restype = c_int32
     lib.fd_scale_by_degree.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_double, c_void_p, c_int64]
     for name in ("fd_synchronize", "fd_create", "fd_destroy", "fd_set_option", "fd_get_option", "fd_beta0", "fd_degree", "fd_apply",
-                 "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_nystrom", "fd_scale_by_degree"):
+                 "fd_apply_general", "fd_eigs", "fd_beta_flow", "fd_beta_flow_cascade", "fd_nystrom", "fd_scale_by_degree"):
         getattr(lib, name).restype = c_int32
     lib.fd_apply_general_static.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_double, c_void_p, c_void_p, c_void_p,
                                             c_int64, c_int32, c_void_p, c_int64, c_void_p, ctypes.c_char_p, c_size_t]
@@ -267,6 +274,32 @@ class Context:
                                   _ptr(U), _ld(U))
         self._check(st)
         recs = [{f[0]: getattr(log[i], f[0]) for f in fd_probe._fields_} for i in range(n.value)]
+        return bx.value, FLOW_OUTCOMES[outcome.value], np.array(ev[:], dtype=np.float64), U, recs
+
+    def beta_flow_cascade(self, k: int, b: int, alpha: float, stages, beta_start: float = 0.0, beta_max: float = 1000.0,
+                          max_applies: int = 2000, warm_start: bool = True, Q0: torch.Tensor | None = None,
+                          max_probes: int = 64):
+        """stages: sequence of (precision, eta, tol) with eta / tol <= 0 for the mode's defaults.
+        Returns (beta_x, outcome name, evals, evecs, [list of probe dicts per stage])."""
+        import numpy as np
+        opts = fd_flow_opts(beta_start, beta_max, 2.0, alpha, 0.0, 0.0, k, b, max_applies, 1 if warm_start else 0)
+        ns = len(stages)
+        st_arr = (fd_cascade_stage * ns)(*[fd_cascade_stage(int(p), float(e), float(t)) for p, e, t in stages])
+        cap = max_probes * ns
+        log = (fd_probe * cap)()
+        n = c_int32(cap)
+        first = (c_int32 * (ns + 1))()
+        outcome = c_int32()
+        bx = c_double()
+        ev = (c_double * (k + 1))()
+        U = _colmajor(self.N, k + 1, self.device)
+        with torch.cuda.device(self.device):
+            st = lib.fd_beta_flow_cascade(self._h, byref(opts), st_arr, ns, _ptr(Q0), 0 if Q0 is None else _ld(Q0),
+                                          0 if Q0 is None else Q0.shape[1], log, byref(n), first, byref(outcome), byref(bx),
+                                          ev, _ptr(U), _ld(U))
+        self._check(st)
+        recs = [[{f[0]: getattr(log[i], f[0]) for f in fd_probe._fields_} for i in range(first[s], first[s + 1])]
+                for s in range(ns)]
         return bx.value, FLOW_OUTCOMES[outcome.value], np.array(ev[:], dtype=np.float64), U, recs
 
     def nystrom(self, Xnew: torch.Tensor, psi: torch.Tensor, evals) -> torch.Tensor:

@@ -87,7 +87,7 @@ struct Solver {
         for (int o = 0; o < cnt; o += bw) {
             int w = std::min(bw, cnt - o);
             FD_TRY(apply_general(c, c->beta, c->s(), c->s(), false, nullptr, N, 0, Q + (int64_t)(c0 + o) * N, N, w,
-                                 W + (int64_t)(c0 + o) * N, N, FD_PREC_FP32, /*gather_out=*/false));
+                                 W + (int64_t)(c0 + o) * N, N, c->eigs_prec, /*gather_out=*/false));
             ++applies;
         }
         FD_TRY(tc_check_status(c));

@@ -64,36 +64,38 @@ double parabola_vertex(const fd_probe& a, const fd_probe& b, const fd_probe& c) 
 
 using namespace fd;
 
-extern "C" fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts* o, const float* Q0_dev, int64_t ldq0, int32_t q0_cols,
-                                  fd_probe* log, int32_t* n_probes, int32_t* outcome, double* beta_x_host,
-                                  double* evals_host, float* evecs_dev, int64_t ldv) {
-    if (!c) return FD_ERR_INVALID;
-    if (!o || !log || !n_probes || *n_probes < 4 || !outcome || !beta_x_host || !evals_host || !evecs_dev)
-        return fail(c, FD_ERR_INVALID, "fd_beta_flow: null argument or log capacity < 4");
-    if (o->k < 1 || !(o->ratio > 1.0) || !(o->beta_max > 0)) return fail(c, FD_ERR_INVALID, "fd_beta_flow: bad options");
-    const int cap = *n_probes;
-    *n_probes = 0;
+namespace fd {
+namespace {
+
+// One sweep of the flow in one precision mode: probes beta_start * ratio^j with the stage's eta and tolerance.
+// log has room for cap records; *n_out receives the number written.
+fd_status flow_stage(fd_ctx* c, const fd_flow_opts* o, fd_precision prec, double eta, double tol, double beta,
+                     const float* Q0_dev, int64_t ldq0, int32_t q0_cols, fd_probe* log, int cap, int32_t* n_out,
+                     int32_t* outcome, double* beta_x_host, double* evals_host, float* evecs_dev, int64_t ldv) {
+    *n_out = 0;
     const int64_t N = c->L.N;
-    const double eta = o->eta > 0 ? o->eta : 1e-7;
-    double beta = o->beta_start;
-    if (!(beta > 0)) FD_TRY(fd_beta0(c, &beta));
     const int k = o->k;
     std::vector<double> lam(k + 1);
     int n = 0;
     bool have_prev = false;
+    struct PrecGuard {                                   // fd_eigs applies M in the stage's mode; restored on every exit
+        fd_ctx* c; fd_precision saved;
+        ~PrecGuard() { c->eigs_prec = saved; }
+    } guard{c, c->eigs_prec};
+    c->eigs_prec = prec;
 
     auto run_probe = [&](double b_, fd_probe& rec, bool warm) -> fd_status {
         rec = fd_probe{};
         rec.beta = b_;
-        FD_TRY(fd_degree(c, b_, o->alpha, FD_PREC_FP32, nullptr, nullptr, nullptr, &rec.S_off, &rec.S_off_2beta));
+        FD_TRY(fd_degree(c, b_, o->alpha, prec, nullptr, nullptr, nullptr, &rec.S_off, &rec.S_off_2beta));
         fd_eigs_info info{};
         const float* q0 = nullptr; int64_t ld0 = 0; int32_t nc0 = 0;
         if (warm && have_prev) { q0 = evecs_dev; ld0 = ldv; nc0 = k + 1; }
         else if (Q0_dev && !have_prev) { q0 = Q0_dev; ld0 = ldq0; nc0 = q0_cols; }
-        fd_status est = fd_eigs(c, k, o->b, o->tol, o->max_applies, q0, ld0, nc0, lam.data(), evecs_dev, ldv, &info);
-        // a probe whose residuals stalled above tol (noise-smeared spectrum at the fp32 floor) still gives eigenvalues
-        // far more accurate than the potential needs: keep it, flagged, if its residuals are below 1e-4
-        if (est == FD_ERR_NOT_CONVERGED && info.max_residual <= 1e-4 * std::fabs(lam[0])) { rec.flags |= 4; est = FD_OK; }
+        fd_status est = fd_eigs(c, k, o->b, tol, o->max_applies, q0, ld0, nc0, lam.data(), evecs_dev, ldv, &info);
+        // a probe whose residuals stalled above tol (noise-smeared spectrum at the operator's accuracy floor) still
+        // gives eigenvalues far more accurate than the potential needs: keep it, flagged, if its residuals are small
+        if (est == FD_ERR_NOT_CONVERGED && info.max_residual <= std::max(1e-4, 100.0 * tol) * std::fabs(lam[0])) { rec.flags |= 4; est = FD_OK; }
         if (est != FD_OK) return est;
         have_prev = true;
         rec.applies = info.applies;
@@ -107,7 +109,7 @@ extern "C" fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts* o, const float*
             FD_TRY(run_probe(bx, tmp, true));
         }
         for (int i = 0; i <= k; ++i) evals_host[i] = lam[i];
-        *beta_x_host = bx; *outcome = oc; *n_probes = n;
+        *beta_x_host = bx; *outcome = oc; *n_out = n;
         return FD_OK;
     };
 
@@ -122,7 +124,7 @@ extern "C" fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts* o, const float*
             for (int i = n - 2; i >= 0; --i)
                 if (!(log[i].flags & 1)) { last_safe = i; break; }
             if (last_safe < 0) {
-                *n_probes = n; *outcome = FD_FLOW_PERRON_WALL; *beta_x_host = NAN;
+                *n_out = n; *outcome = FD_FLOW_PERRON_WALL; *beta_x_host = NAN;
                 return fail(c, FD_ERR_PERRON_WALL, "first probe already at the Perron wall (g_P = %.3e)", rec.g_P);
             }
             return finish(log[last_safe].beta, FD_FLOW_PERRON_WALL, true);
@@ -140,6 +142,60 @@ extern "C" fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts* o, const float*
     }
     if (n == 0) return fail(c, FD_ERR_INVALID, "fd_beta_flow: beta_start beyond beta_max");
     return finish(log[n - 1].beta, FD_FLOW_RIGHT_EDGE, false);
+}
+
+}  // namespace
+}  // namespace fd
+
+extern "C" fd_status fd_beta_flow(fd_ctx* c, const fd_flow_opts* o, const float* Q0_dev, int64_t ldq0, int32_t q0_cols,
+                                  fd_probe* log, int32_t* n_probes, int32_t* outcome, double* beta_x_host,
+                                  double* evals_host, float* evecs_dev, int64_t ldv) {
+    if (!c) return FD_ERR_INVALID;
+    if (!o || !log || !n_probes || *n_probes < 4 || !outcome || !beta_x_host || !evals_host || !evecs_dev)
+        return fail(c, FD_ERR_INVALID, "fd_beta_flow: null argument or log capacity < 4");
+    if (o->k < 1 || !(o->ratio > 1.0) || !(o->beta_max > 0)) return fail(c, FD_ERR_INVALID, "fd_beta_flow: bad options");
+    const int cap = *n_probes;
+    double beta = o->beta_start;
+    if (!(beta > 0)) FD_TRY(fd_beta0(c, &beta));
+    return flow_stage(c, o, FD_PREC_FP32, o->eta > 0 ? o->eta : 1e-7, o->tol, beta, Q0_dev, ldq0, q0_cols, log, cap, n_probes,
+                      outcome, beta_x_host, evals_host, evecs_dev, ldv);
+}
+
+extern "C" fd_status fd_beta_flow_cascade(fd_ctx* c, const fd_flow_opts* o, const fd_cascade_stage* stages, int32_t n_stages,
+                                          const float* Q0_dev, int64_t ldq0, int32_t q0_cols, fd_probe* log,
+                                          int32_t* n_probes, int32_t* stage_first_probe, int32_t* outcome,
+                                          double* beta_x_host, double* evals_host, float* evecs_dev, int64_t ldv) {
+    if (!c) return FD_ERR_INVALID;
+    if (!o || !stages || n_stages < 1 || n_stages > 8 || !log || !n_probes || *n_probes < 4 * n_stages || !stage_first_probe ||
+        !outcome || !beta_x_host || !evals_host || !evecs_dev)
+        return fail(c, FD_ERR_INVALID, "fd_beta_flow_cascade: null argument, bad stage count or log capacity < 4 per stage");
+    if (o->k < 1 || !(o->ratio > 1.0) || !(o->beta_max > 0)) return fail(c, FD_ERR_INVALID, "fd_beta_flow_cascade: bad options");
+    for (int s = 0; s < n_stages; ++s)
+        if (stages[s].prec != FD_PREC_FP32 && stages[s].prec != FD_PREC_FAST) return fail(c, FD_ERR_INVALID, "fd_beta_flow_cascade: bad precision");
+    const int cap = *n_probes;
+    int used = 0;
+    *n_probes = 0;
+    double beta = o->beta_start;
+    if (!(beta > 0)) FD_TRY(fd_beta0(c, &beta));
+    for (int s = 0; s < n_stages; ++s) {
+        const bool fast = stages[s].prec == FD_PREC_FAST;
+        const double eta = stages[s].eta > 0 ? stages[s].eta : (fast ? 1e-3 : 1e-7);
+        const double tol = stages[s].tol > 0 ? stages[s].tol : (fast ? 1e-3 : 1e-6);
+        stage_first_probe[s] = used;
+        int32_t n_stage = 0;
+        // the first stage starts from the caller's basis, every later one from the previous stage's eigenvectors
+        const float* q0 = s == 0 ? Q0_dev : evecs_dev;
+        const int64_t ld0 = s == 0 ? ldq0 : ldv;
+        const int32_t nc0 = s == 0 ? q0_cols : o->k + 1;
+        fd_status st = flow_stage(c, o, stages[s].prec, eta, tol, beta, q0, ld0, nc0, log + used, cap - used, &n_stage, outcome,
+                                  beta_x_host, evals_host, evecs_dev, ldv);
+        used += n_stage;
+        *n_probes = used;
+        stage_first_probe[s + 1] = used;
+        if (st != FD_OK) return st;
+        beta = *beta_x_host / o->ratio;                  // the next stage restarts one grid step below this selection
+    }
+    return FD_OK;
 }
 
 extern "C" fd_status fd_nystrom(fd_ctx* c, const float* Xnew_dev, int64_t Nnew, int64_t ldxnew, const float* psi_dev,

@@ -57,6 +57,7 @@ struct fd_ctx {
     int opt_flush = 0;
     int opt_jt_chunk = 0;            // column tiles per L2-resident chunk of the tensor-core block product (0 = default)
     int last_path = 0;               // kernel family that served the most recent quadratic pass (FD_PATH_SIMT / FD_PATH_TC)
+    fd_precision eigs_prec = FD_PREC_FP32;   // precision mode of fd_eigs's block products (set per stage by the cascade)
     double opt_tc_max_mag = 72.0;    // largest beta' * max|x - mu|^2 the Gram-form kernel is trusted with in fp32 mode
     std::string err;
     // pinned host staging ring for the eigensolver's small uploads (allocated on the first fd_eigs, freed by fd_destroy:

@@ -319,3 +319,62 @@ def test_beta_flow_edge_outcomes_match_oracle(fd, dev, beta_start, beta_max, exp
     lam_o, _, _ = dense.eigs(X, bx_o, alpha, k)
     assert np.abs(lam - lam_o).max() <= 1e-6
     ctx.close()
+
+
+# ------------------------------------------------------------------ precision cascade (Sec. 2.3, last paragraph)
+def test_precision_cascade_matches_oracle_cascade(fd, dev):
+    """Reduced-precision sweep first (eta = 1e-3 in Eqs. 11-12), then the fp32 sweep restarted one grid step below its
+    selection.  The oracle runs the same two stages in float64 (the data type enters it only through eta).  Stage 1
+    is compared loosely (the reduced-precision operator is 2e-4 away from the exact one); stage 2 probe by probe at the
+    fp32 gates, from the bandwidth the GPU's own stage 1 selected."""
+    N, alpha, k = 2048, 0.5, 3
+    X = workloads.torus6_paper(N, seed=42)
+    probe = flow.dense_probe(X, alpha, k)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    ctx.set_option("path", fd.FD_PATH_TC)              # the reduced-precision mode exists on the Gram-form kernels only
+    bx, status, lam, U, stages = ctx.beta_flow_cascade(k, 8, alpha, [(fd.FD_PREC_FAST, 0.0, 0.0), (fd.FD_PREC_FP32, 0.0, 0.0)])
+    assert len(stages) == 2 and status == "VERTEX"
+    # stage 1 against the oracle's eta = 1e-3 sweep
+    bx1_o, st1_o, log1_o = flow.beta_flow(probe, N, flow.beta0(X), 1000.0, eta=1e-3)
+    s1 = stages[0]
+    assert len(s1) == len(log1_o) and st1_o == "VERTEX"
+    for r, ro in zip(s1[:-1], log1_o[:-1]):
+        assert r["beta"] == pytest.approx(ro["beta"], rel=1e-6)
+        assert r["V"] == pytest.approx(ro["V"], rel=2e-2)
+        assert r["V_mach"] == pytest.approx(ro["V_mach"], rel=0.2, abs=1e-6)      # (10 eta / g_P)^6 with the stage's eta
+    bx1 = s1[-1]["beta"]
+    assert bx1 == pytest.approx(bx1_o, rel=3e-2)
+    # stage 2 = the fp32 flow from bx1 / 2: probe by probe against the oracle started at the same point
+    bx2_o, st2_o, log2_o = flow.beta_flow(probe, N, bx1 / 2.0, 1000.0, eta=1e-7)
+    s2 = stages[1]
+    assert s2[0]["beta"] == pytest.approx(bx1 / 2.0, rel=1e-12)
+    assert len(s2) == len(log2_o) and st2_o == "VERTEX"
+    for r, ro in zip(s2, log2_o):
+        assert r["beta"] == pytest.approx(ro["beta"], rel=1e-3)
+        assert r["V"] == pytest.approx(ro["V"], rel=1e-3)
+    assert bx == pytest.approx(bx2_o, rel=1e-3)
+    check_eigs(lam, U.cpu().numpy(), X, bx, alpha, k, angle_gate=True)
+    assert ctx.get_option("beta") == pytest.approx(bx)
+    # the whole cascade agrees with the oracle's own two-stage run to the accuracy stage 1 allows
+    bx_c, st_c, logs_c = flow.cascade([probe, probe], N, flow.beta0(X), 1000.0, [1e-3, 1e-7])
+    assert st_c == "VERTEX" and bx == pytest.approx(bx_c, rel=3e-2)
+    # the cascade spends fewer fp32-mode applies than the fp32-only flow
+    ctx2 = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    ctx2.set_option("path", fd.FD_PATH_TC)
+    bx_f, st_f, lam_f, U_f, recs_f = ctx2.beta_flow(k, 8, alpha, beta_start=0.0, beta_max=1000.0)
+    assert sum(r["applies"] for r in s2) < sum(r["applies"] for r in recs_f)
+    assert bx == pytest.approx(bx_f, rel=0.1)
+    ctx.close(); ctx2.close()
+
+
+def test_cascade_single_fp32_stage_is_the_plain_flow(fd, dev):
+    N, alpha, k = 1024, 0.5, 3
+    X = workloads.torus6_paper(N, seed=42)
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8, m_max=64)
+    bx, status, lam, U, recs = ctx.beta_flow(k, 8, alpha, beta_start=0.0, beta_max=1000.0)
+    bx_c, status_c, lam_c, U_c, stages = ctx.beta_flow_cascade(k, 8, alpha, [(fd.FD_PREC_FP32, 1e-7, 1e-6)])
+    assert (bx_c, status_c) == (bx, status) and np.array_equal(lam, lam_c)
+    assert [r["beta"] for r in stages[0]] == [r["beta"] for r in recs]
+    with pytest.raises(fd.FdError):
+        ctx.beta_flow_cascade(k, 8, alpha, [])
+    ctx.close()
