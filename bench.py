@@ -488,6 +488,7 @@ def time_to_k_eigs(fd, dev, args, transport=None):
     if not args.eigs_case and transport is None:
         res.append(ladder(fd, dev, args.ladder_full))
         res.append({"t6_validation": t6_validation(fd, dev, args.t6_full)})
+        res.append({"paper_shape_context": paper_shape_context(fd, dev)})
     return res
 
 
@@ -534,6 +535,38 @@ def t6_validation(fd, dev, full=False):
         if N in printed:
             rec["printed_beta_x"], rec["printed_one_minus_overlap"] = printed[N][0], 1.0 - printed[N][1]
         out.append(rec)
+    return out
+
+
+def paper_shape_context(fd, dev):
+    """Context rows: the raw kernel application K V on the paper's own race shape (App. B: anisotropic T^6 zero-padded to
+    D = 32, beta = 1, b = 1 and b = 8), fp32-grade mode, with the times the paper prints for its kernel on another GPU
+    (RTX PRO 6000) beside them.  Not the metric's configuration and not a target: context."""
+    import torch
+    import workloads
+    printed = {(1 << 17, 1): 0.03901, (1 << 17, 8): 0.04319, (1 << 20, 1): 2.083, (1 << 20, 8): 2.897}
+    out = []
+    for e in (17, 20):
+        N = 1 << e
+        X = torch.from_numpy(workloads.torus6_paper(N, seed=42)).to(dev)
+        ctx = fd.Context(X, b_max=8, m_max=0)
+        for b in (1, 8):
+            V = torch.from_numpy(np.ascontiguousarray(workloads.block(N, b, seed=7).T)).to(dev).t()
+            Y = torch.empty((b, N), dtype=torch.float32, device=dev).t()
+            ctx.apply_general(1.0, V, out=Y)
+            torch.cuda.synchronize(dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = 3
+            e0.record()
+            for _ in range(reps):
+                ctx.apply_general(1.0, V, out=Y)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            t = e0.elapsed_time(e1) / reps * 1e-3
+            out.append({"N": N, "D": 32, "beta": 1.0, "b": b, "seconds": t, "pair_cols_per_s": float(N) * N * b / t,
+                        "path": "tc" if ctx.get_option("last_path") == 2 else "simt",
+                        "printed_seconds_other_gpu": printed[(N, b)]})
+        ctx.close()
     return out
 
 
