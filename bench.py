@@ -448,7 +448,7 @@ def time_to_k_eigs(fd, dev, args, transport=None):
             Xnp = Xc
         N = Xnp.shape[0]
         X = torch.from_numpy(Xnp).to(dev)
-        m_max = default_m_max(k, b)
+        m_max = args.m_max if args.m_max > 0 else default_m_max(k, b)
         ctx = fd.Context(X, b_max=b, m_max=m_max)
         if transport is not None:
             ctx.set_shard(fd.Shard(transport, N, b, dev))
@@ -462,7 +462,7 @@ def time_to_k_eigs(fd, dev, args, transport=None):
         rec = {"workload": f"{name}: N={N}, D={Xnp.shape[1]}, k={k}, b={b}, alpha=1, beta={beta}, tol=1e-6",
                "path": "tc" if ctx.get_option("last_path") == 2 else "simt", "degree_s": t1 - t0,
                "eigs_s": t2 - t1, "total_s": t2 - t0, "applies": int(info.applies), "restarts": int(info.restarts),
-               "converged": int(info.converged), "of": k + 1, "max_residual": float(info.max_residual),
+               "converged": int(info.converged), "of": k + 1, "max_residual": float(info.max_residual), "m_max": m_max,
                "seconds_in_apply": float(info.seconds_apply), "lambda_1": float(lam[1]), "lambda_k": float(lam[k])}
         if name.startswith("C3"):
             t3 = time.perf_counter()
@@ -508,6 +508,7 @@ def t6_validation(fd, dev, full=False):
                     printed[int(r[0])] = (float(r[1]), float(r[3]))
     except OSError:
         pass
+    printed_s = {1024: 6.03, 16384: 6.37, 65536: 15.98, 131072: 61.58, 262144: 147.90, 524288: 464.25, 1048576: 2225.04}
     out = []
     for e in range(10, 21 if full else 18):
         N = 1 << e
@@ -534,6 +535,8 @@ def t6_validation(fd, dev, full=False):
                "flow_s": dt, "path": path, "n_eff": recs[-1]["n_eff"], "d_hat": recs[-1]["d_hat"], "one_minus_overlap": 1.0 - score}
         if N in printed:
             rec["printed_beta_x"], rec["printed_one_minus_overlap"] = printed[N][0], 1.0 - printed[N][1]
+        if N in printed_s:
+            rec["printed_time_to_solution_s_other_gpu"] = printed_s[N]     # Fig. 1(a): flow + ladder + solver, one RTX PRO 6000
         out.append(rec)
     return out
 
@@ -571,9 +574,11 @@ def paper_shape_context(fd, dev):
 
 
 def default_m_max(k, b):
-    """Basis capacity for fd_eigs: room for the wanted pairs twice over plus one block, at least four blocks, and at least
-    64 columns (a very small capacity forces a thick restart on almost every step)."""
-    return (max(2 * (k + 1) + b, 4 * b, min(8 * b, 64)) + b - 1) // b * b
+    """Basis capacity for fd_eigs: three times the wanted pairs plus two blocks, at least four blocks and at least 64
+    columns.  The thick restart keeps 3/5 of the capacity, so this keeps about twice the wanted pairs: room for the rest
+    of an eigenvalue cluster that the request cuts (the 6-torus at k = 128 cuts a 160-fold cluster: with room for it all
+    129 pairs converge in 44 block products, with 2 (k + 1) + b columns only 73 do in 125)."""
+    return (max(3 * (k + 1) + 2 * b, 4 * b, 64) + b - 1) // b * b
 
 
 def ladder(fd, dev, full=False):
@@ -652,6 +657,7 @@ def main():
     ap.add_argument("--no-c5-eigs", action="store_true", help="skip the eigensolve at N = 2^20 (k = 128, b = 64; about 80 s)")
     ap.add_argument("--eigs-case", default="", choices=["", "C1", "C2", "C3", "C4", "C5"],
                     help="time-to-k-eigenpairs leg: only this configuration (and no ladder)")
+    ap.add_argument("--m-max", type=int, default=0, help="basis capacity of the eigensolver legs (0: default_m_max(k, b))")
     ap.add_argument("--t6-full", action="store_true", help="T^6 validation sweep up to N = 2^20 instead of 2^17")
     ap.add_argument("--ladder-full", action="store_true", help="run config 5's own ladder (2^16 ... 2^20, k = 128, b = 64; many minutes)")
     args = ap.parse_args()

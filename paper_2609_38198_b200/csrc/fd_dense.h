@@ -23,9 +23,10 @@ fd_status random_fill(fd_ctx* c, float* A, int64_t lda, int p, int64_t N, int64_
 fd_status sqrt_vec(fd_ctx* c, const float* d, float* out, int64_t N);
 fd_status copy_cols(fd_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd, int p, int64_t N);
 
-// Eigen-decomposition of a dense symmetric n x n matrix (column-major, only read).  On return
-// evals ascending and evecs column-major with orthonormal columns.  Householder tridiagonalisation
-// followed by implicit-shift QL.  Returns false if QL fails to converge.
-bool sym_eig(const double* A, int n, std::vector<double>& evals, std::vector<double>& evecs);
+// Eigen-decomposition of a dense symmetric n x n matrix (column-major, only read).  On return evals ascending (all n) and
+// evecs n x n column-major with orthonormal columns; with 0 <= nvec < n only the columns of the nvec LARGEST eigenvalues
+// (columns n - nvec .. n - 1) are computed, the others are zero.  Householder tridiagonalisation followed by implicit
+// symmetric QR.  Returns false if the iteration fails to converge.
+bool sym_eig(const double* A, int n, std::vector<double>& evals, std::vector<double>& evecs, int nvec = -1);
 
 }  // namespace fd

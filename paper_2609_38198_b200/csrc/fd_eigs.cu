@@ -294,7 +294,10 @@ extern "C" fd_status fd_eigs(fd_ctx* c, int32_t k, int32_t b, double tol, int32_
                 Tc[i + (size_t)j * m] = S.T[i + (size_t)j * m_cap] - 0.5 * (ET[i + (size_t)j * m] + ET[j + (size_t)i * m]);
         std::vector<double> lam, U;
         auto tp1 = clk::now();
-        if (!sym_eig(Tc.data(), m, lam, U)) return fail(c, FD_ERR_NOT_CONVERGED, "projected eigenproblem failed");
+        // eigenvectors: the leading Ritz vectors on every step; the larger kept set only when this step may restart
+        const int nvec_ritz = std::min(nsel_max, m);
+        const int nvec = (m + b > m_cap) ? std::max(nvec_ritz, std::min(m - 1, (m_cap * 3) / 5)) : nvec_ritz;
+        if (!sym_eig(Tc.data(), m, lam, U, nvec)) return fail(c, FD_ERR_NOT_CONVERGED, "projected eigenproblem failed");
         auto tp2 = clk::now();
         t_rr += secs(tp0, tp1); t_eig += secs(tp1, tp2);
         nsel = std::min(nsel_max, m);

@@ -21,7 +21,7 @@
 // One persistent CTA per SM: warps 0-3 / 4-7 = the two exponential warpgroups (raised to 232 registers);
 // warp 8 = TMA producer, warps 9 / 10 = product-MMA issuers for row tile 0 / 1, warp 11 = Gram-MMA issuer
 // (lowered to 40 registers).  Three issuing threads because the per-tile bookkeeping of a lone issuer
-// (waits, commits, descriptors) cost about as much as its MMAs and left the tensor pipe idle.  Column tiles are staged by TMA (no multicast) through a 4-deep ring.
+// (waits, commits, descriptors) cost about as much as its MMAs and left the tensor pipe idle.  Column tiles are staged by TMA (every CTA loads its own copy) through a 4-deep ring.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains and exits.
 #include <cuda.h>
 

@@ -17,7 +17,7 @@
 //                tensor core, so neither the MUFU (four warps per scheduler, in different phases) nor the tensor pipe
 //                waits for the other in steady state;
 //   warps 16-19  flush warpgroup: owns the fp32 accumulator registers and the epilogue;
-//   warp 20      TMA producer (4-stage ring of column tiles, no multicast);
+//   warp 20      TMA producer (4-stage ring of column tiles; every CTA loads its own copy);
 //   warp 21 / 22 product-MMA issuer / Gram-MMA issuer (one thread each: two independent dependency chains).
 // TMEM (512 columns): three S/P buffers at [0, 384), accumulator at [384, 384 + BT).
 // Registers: compiled for 80 per thread (65536 / 768 rounded down to the allocation unit); setmaxnreg then moves
