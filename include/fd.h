@@ -147,7 +147,11 @@ typedef struct {
  * implicitly restarted Lanczos and gives no further detail; Sec. 2.3).  b = block size,
  * tol = residual tolerance relative to theta_0, Q0_dev = optional warm-start basis (N x q0_cols,
  * need not be orthonormal).  evals_host: k + 1 doubles, descending.  evecs_dev: N x (k + 1)
- * column-major, orthonormal.  Needs m_max >= 2 (k + 1) + b at fd_create.  Synchronous. */
+ * column-major, orthonormal.  Needs m_max >= 2 (k + 1) + b at fd_create; the thick restart keeps 3/5 of m_max, so a
+ * capacity near 3 (k + 1) + 2 b keeps room for the rest of an eigenvalue cluster that the request cuts (on the
+ * 6-torus, k = 128 cuts a 160-fold cluster: 129 of 129 pairs converge in 43 block products with m_max = 576, 73 of
+ * 129 in 125 with 384).  info->converged counts the LEADING pairs below tol.  On FD_ERR_NOT_CONVERGED the outputs hold
+ * the best current Ritz pairs.  Synchronous. */
 fd_status fd_eigs(fd_ctx* ctx, int32_t k, int32_t b, double tol, int32_t max_applies,
                   const float* Q0_dev, int64_t ldq0, int32_t q0_cols,
                   double* evals_host, float* evecs_dev, int64_t ldv, fd_eigs_info* info);
