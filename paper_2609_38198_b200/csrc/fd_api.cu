@@ -63,6 +63,7 @@ Layout make_layout(int64_t N, int32_t D, int32_t b_max, int32_t m_max) {
     L.wt_lo = carve(cur, (size_t)L.BP * L.NP * 2);
     L.colscale = carve(cur, (size_t)(L.BP + 8) * 4 * 2);
     L.status = carve(cur, 256);
+    L.symsum = carve(cur, (size_t)N * 8);
     if (m_max > 0) {
         L.eig_q = carve(cur, (size_t)N * m_max * 4);
         L.eig_w = carve(cur, (size_t)N * m_max * 4);
@@ -155,6 +156,9 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "flush")) {
         if (v < 0 || v > 1 << 20) return fail(c, FD_ERR_INVALID, "flush out of range");
         c->opt_flush = (int)v;
+    } else if (!strcmp(name, "sym")) {
+        if (v != 0 && v != 1) return fail(c, FD_ERR_INVALID, "sym must be 0 or 1");
+        c->opt_sym = (int)v;
     } else if (!strcmp(name, "jt_chunk")) {
         if (v < 0 || v > 1 << 24) return fail(c, FD_ERR_INVALID, "jt_chunk out of range");
         c->opt_jt_chunk = (int)v;
@@ -175,6 +179,7 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     if (!strcmp(name, "path")) *v = c->opt_path;
     else if (!strcmp(name, "splits")) *v = c->opt_splits;
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
+    else if (!strcmp(name, "sym")) *v = c->opt_sym;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "last_path")) *v = c->last_path;
     else if (!strcmp(name, "tc_cycles")) {
@@ -213,6 +218,7 @@ fd_status fd_degree(fd_ctx* c, double beta, double alpha, fd_precision prec, flo
     a.xrow = c->xs() + r0 * c->L.DP; a.Nrow = n; a.rows_are_ctx = true; a.beta = beta;
     a.left = nullptr; a.right = nullptr; a.V = nullptr; a.ldv = N; a.b = 1;
     a.Y = c->q() + r0; a.ldy = N; a.rowsq = rowsq + r0; a.prec = prec;
+    a.sym_ok = !c->sh.on;                                        // K = K^T, unit weights
     if (n > 0) FD_TRY(apply_dispatch(c, a));
     double sums[2] = {0.0, 0.0};
     if (n > 0) FD_TRY(reduce_sums(c, c->q() + r0, rowsq + r0, n, &sums[0], &sums[1]));
@@ -228,7 +234,7 @@ fd_status fd_degree(fd_ctx* c, double beta, double alpha, fd_precision prec, flo
         // pass 2: d = q^-alpha * K q^-alpha
         FD_TRY(ew_pow(c, c->q(), -alpha, c->w(), N));
         ApplyArgs a2 = a;
-        a2.left = c->w() + r0; a2.right = c->w(); a2.Y = c->d() + r0; a2.rowsq = nullptr; a2.right_pos = true;
+        a2.left = c->w() + r0; a2.right = c->w(); a2.Y = c->d() + r0; a2.rowsq = nullptr; a2.right_pos = true;       // (sym_ok stays: left = right = q^-alpha in (0, 1])
         if (n > 0) FD_TRY(apply_dispatch(c, a2));
         FD_TRY(gather_rows(c, c->d(), N, 1));
         FD_TRY(ew_scale_vec(c, c->w(), c->d(), c->s(), N));

@@ -30,6 +30,7 @@ struct Layout {
     size_t wp = 0, part = 0, part_floats = 0;
     size_t xp_col = 0, xp_row = 0, wt_hi = 0, wt_lo = 0, colscale = 0, status = 0;
     size_t yacc = 0;
+    size_t symsum = 0;               // N 64-bit fixed-point sums of the symmetric row-sum mode
     size_t eig_q = 0, eig_w = 0, eig_x = 0, eig_r = 0, eig_t = 0, eig_small = 0, eig_small_doubles = 0;
     size_t total = 0;
 };
@@ -55,6 +56,7 @@ struct fd_ctx {
     int opt_path = FD_PATH_AUTO;
     int opt_splits = 0;
     int opt_flush = 0;
+    int opt_sym = 1;                 // symmetric half-work degree passes on the Gram-form kernels (0 = evaluate every tile)
     int opt_jt_chunk = 0;            // column tiles per L2-resident chunk of the tensor-core block product (0 = default)
     int last_path = 0;               // kernel family that served the most recent quadratic pass (FD_PATH_SIMT / FD_PATH_TC)
     fd_precision eigs_prec = FD_PREC_FP32;   // precision mode of fd_eigs's block products (set per stage by the cascade)
@@ -125,6 +127,7 @@ struct ApplyArgs {
     float* Y; int64_t ldy;
     double* rowsq;                          // optional: sum_j K_ij^2 per row (rowsum mode, b = 1, V null)
     bool right_pos;                         // caller guarantees right > 0 elementwise
+    bool sym_ok;                            // square pass with left == right, weights in (0, 1]: the symmetric half-work row sums may serve it
     fd_precision prec;
 };
 fd_status apply_simt(fd_ctx* c, const ApplyArgs& a);

@@ -40,11 +40,13 @@ using namespace tc;
 template <int BT, int MODE>
 struct Smem {
     static constexpr int kXChunk = 128 * 64;                       // one K slab (hi|lo) of 128 points: 8 KB
-    static constexpr int kWHalf = (MODE == kModeRowsum) ? 0 : BT * 128;   // 64 j x BT columns fp16
-    static constexpr int kWBytes = (MODE == kModeRowsum) ? 0 : 4 * kWHalf;   // [W_hi j-half 0][W_hi j-half 1][W_lo 0][W_lo 1]
+    static constexpr int kWHalf = is_rowsum(MODE) ? 0 : BT * 128;   // 64 j x BT columns fp16
+    static constexpr int kWBytes = is_rowsum(MODE) ? 0 : 4 * kWHalf;   // [W_hi j-half 0][W_hi j-half 1][W_lo 0][W_lo 1]
+    // symmetric row-sum mode: per-warp column partial sums, [row tile][parity][warp quarter][128 columns] floats
+    static constexpr int kColPartBytes = (MODE == kModeRowsumSym) ? 2 * 2 * 4 * 128 * 4 : 0;
     static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
     static __host__ __device__ constexpr int total(int K16) {
-        return 1024 /*align slack*/ + kStages * stage_bytes(K16) + 2 * K16 * kXChunk + 1024 /*barriers*/;
+        return 1024 /*align slack*/ + kStages * stage_bytes(K16) + 2 * K16 * kXChunk + 1024 /*barriers*/ + kColPartBytes;
     }
 };
 
@@ -62,6 +64,7 @@ struct Barriers {
     uint64_t p_half[kMaxBuf][2];            // block mode: first 64 columns of P written (lets the product MMA start early)
     uint64_t kw_done[kMaxBuf][2];           // block mode: product MMAs that read P from this buffer have completed
     uint64_t y_full[2], y_empty[2];         // accumulator flush hand-off (per row tile)
+    uint64_t col_ready[2][2];               // symmetric row-sum mode: the four warps' column partials of a tile are written
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -76,7 +79,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
      const __grid_constant__ CUtensorMap map_whi, const __grid_constant__ CUtensorMap map_wlo, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using SM = Smem<BT, MODE>;
-    constexpr int NBUF = (MODE == kModeRowsum) ? 4 : 3;
+    constexpr int NBUF = is_rowsum(MODE) ? 4 : 3;
     constexpr uint32_t kRingPeriod = (NBUF & 1) ? 2 * NBUF : NBUF;   // tiles between two uses of a buffer by the same row tile
     constexpr uint32_t kYCol = 384;                    // block mode: Y_t at columns 384 + 64 t
     const int K16 = p.K16;
@@ -90,7 +93,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
 
     if (threadIdx.x == 0) {
         // a column stage is released by the Gram issuer alone (row-sum mode) or by both product issuers (block mode)
-        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], MODE == kModeRowsum ? 1 : 2); }
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], is_rowsum(MODE) ? 1 : 2); }
         mbar_init(&bars->xfull, 1); mbar_init(&bars->xempty, 1);
         for (int u = 0; u < kMaxBuf; ++u)
             for (int t = 0; t < 2; ++t) {
@@ -98,6 +101,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 mbar_init(&bars->kw_done[u][t], 1); mbar_init(&bars->p_half[u][t], 4);
             }
         for (int t = 0; t < 2; ++t) { mbar_init(&bars->y_full[t], 1); mbar_init(&bars->y_empty[t], 4); }
+        for (int t = 0; t < 2; ++t)
+            for (int u = 0; u < 2; ++u) mbar_init(&bars->col_ready[t][u], 4);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -114,13 +119,23 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     // Work items of this CTA: (column chunk c, row-pair tile r) with c outermost, r = blockIdx.x + k * gridDim.x.  Every CTA
     // sweeps chunk c for all of its rows before chunk c + 1, so the whole grid reads the same L2-sized slice of the
     // column operands at about the same time; a row's partial results always come from the same threads, in order.
-    const int my_rows = (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_items = my_rows * p.num_chunks;
+    //
+    // Symmetric row-sum mode: only tiles on or above the diagonal are evaluated.  Row pair r needs column tiles 2 r .. num_jt - 1;
+    // pairing r with num_work - 1 - r gives every CTA work units of equal length (num_jt + 2 tiles): unit u = blockIdx.x +
+    // k * gridDim.x is the two items {u, num_work - 1 - u} (the middle pair of an odd count stands alone: its second
+    // item is empty).
+    constexpr bool kSym = MODE == kModeRowsumSym;
+    const int sym_units = (p.num_work + 1) / 2;
+    const int my_rows = kSym ? (sym_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
+                             : (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_items = kSym ? 2 * my_rows : my_rows * p.num_chunks;
 #define FD_ITEM_GEOMETRY(w)                                                                         \
-    const int cch = (w) / my_rows;                                                                  \
-    const int item = (int)blockIdx.x + ((w) % my_rows) * (int)gridDim.x;                            \
-    const int j0 = cch * p.jt_chunk;                                                                \
-    const int num_jt = (p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk;                   \
+    const int unit_ = (int)blockIdx.x + (kSym ? ((w) >> 1) : ((w) % my_rows)) * (int)gridDim.x;     \
+    const int cch = kSym ? 0 : (w) / my_rows;                                                       \
+    const int item = (kSym && ((w) & 1)) ? p.num_work - 1 - unit_ : unit_;                          \
+    const int j0 = kSym ? 2 * item : cch * p.jt_chunk;                                              \
+    const int num_jt = kSym ? ((((w) & 1) && item == unit_) ? 0 : p.num_jt - j0)                    \
+                            : ((p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk);          \
     const int tiles_per_item = 2 * num_jt;                                                          \
     (void)item; (void)tiles_per_item; (void)cch
     const int flush = p.flush;
@@ -131,7 +146,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         // =============================================================== TMA producer (one thread)
         if (lane == 0) {
             prefetch_tmap(&map_xrow); prefetch_tmap(&map_xcol);
-            if (MODE != kModeRowsum) { prefetch_tmap(&map_whi); prefetch_tmap(&map_wlo); }
+            if (!is_rowsum(MODE)) { prefetch_tmap(&map_whi); prefetch_tmap(&map_wlo); }
             uint32_t it = 0;
             bool ok = true;
             for (int w = 0; w < my_items && ok; ++w) {
@@ -151,7 +166,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     mbar_expect_tx(&bars->full[s], SM::stage_bytes(K16));
                     for (int c = 0; c < K16; ++c)
                         tma_load_2d(st + c * SM::kXChunk, &map_xcol, 0, (int)(c * p.np_cols + (int64_t)(j0 + j) * 128), &bars->full[s]);
-                    if (MODE != kModeRowsum) {
+                    if (!is_rowsum(MODE)) {
                         uint8_t* wst = st + K16 * SM::kXChunk;
                         tma_load_2d(wst, &map_whi, (j0 + j) * 128, 0, &bars->full[s]);
                         tma_load_2d(wst + SM::kWHalf, &map_whi, (j0 + j) * 128 + 64, 0, &bars->full[s]);
@@ -173,7 +188,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         // =============================================================== Gram MMA issuer (one thread)
         // Issues S(n) = A_t B_j^T for every tile as soon as its ring buffer is free again; runs up to NBUF tiles ahead.
         if (lane == 0) {
-          if constexpr (MODE == kModeRowsum) {
+          if constexpr (is_rowsum(MODE)) {
             // Row-sum mode: the MUFU binds and the tensor pipe is mostly idle; descriptors are rebuilt per MMA, which paces
             // the Gram MMAs between the warpgroups' TMEM loads (issuing them in tight bursts measured 5 % slower).
             constexpr uint32_t idesc_g = idesc_f16(128);
@@ -192,7 +207,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     if (g >= (uint32_t)NBUF) {
                         // the tile that used this buffer last (NBUF tiles ago, possibly of the other row tile) must be finished
                         const uint32_t gp = g - NBUF;
-                        uint64_t* fb = (MODE == kModeRowsum) ? &bars->s_done[buf][gp & 1] : &bars->kw_done[buf][gp & 1];
+                        uint64_t* fb = is_rowsum(MODE) ? &bars->s_done[buf][gp & 1] : &bars->kw_done[buf][gp & 1];
                         ok = mbar_wait(fb, (gp / kRingPeriod) & 1, abort_flag, p.status, 5);
                         if (!ok) break;
                     }
@@ -206,19 +221,22 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     const uint32_t s_addr = tmem + 128u * buf;
                     const int t = n & 1;
                     uint8_t* st = stage_base + s * SM::stage_bytes(K16);
+                    // (symmetric mode: the streamed tile is the M operand, so TMEM lanes = streamed points)
                     for (int c = 0; c < K16; ++c) {
-                        const uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
-                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
+                        uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        if (MODE == kModeRowsumSym) { const uint64_t x = a; a = b; b = x; }
                         mma_ss(s_addr, a, b + 2, idesc_g, c > 0);          // + 2: the lo half starts 32 B into the row
                         mma_ss(s_addr, a + 2, b, idesc_g, 1);
                     }
                     for (int c = 0; c < K16; ++c) {
-                        const uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
-                        const uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        uint64_t a = smem_desc(smem_u32(xi_base + (t * K16 + c) * SM::kXChunk), 512, 4);
+                        uint64_t b = smem_desc(smem_u32(st + c * SM::kXChunk), 512, 4);
+                        if (MODE == kModeRowsumSym) { const uint64_t x = a; a = b; b = x; }
                         mma_ss(s_addr, a, b, idesc_g, 1);
                     }
                     tc_commit(&bars->s_full[buf][n & 1]);
-                    if (MODE == kModeRowsum && (n & 1)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
+                    if (is_rowsum(MODE) && (n & 1)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
                 }
                 if (ok) tc_commit(&bars->xempty);                  // the row operand tiles may be replaced
                 it0 += (uint32_t)num_jt;
@@ -248,7 +266,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         // the tile that used this buffer last (NBUF tiles ago, possibly of the other row tile) must be finished
                         const int tp = (NBUF & 1) ? (t ^ 1) : t;
                         const uint32_t php = gr >= (uint32_t)NBUF ? ph : ph ^ 1u;
-                        uint64_t* fb = (MODE == kModeRowsum) ? &bars->s_done[buf][tp] : &bars->kw_done[buf][tp];
+                        uint64_t* fb = is_rowsum(MODE) ? &bars->s_done[buf][tp] : &bars->kw_done[buf][tp];
                         ok = mbar_wait(fb, php, abort_flag, p.status, 5);
                         if (!ok) break;
                     }
@@ -277,7 +295,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     }
                     tc_commit(&bars->s_full[buf][t]);
                     if (t == 1) {
-                        if (MODE == kModeRowsum) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
+                        if (is_rowsum(MODE)) tc_commit(&bars->empty[s]);   // both Gram MMAs of this column tile issued
                         ++itj;
                     }
                     if (++buf == (uint32_t)NBUF) { buf = 0; first_round = false; }
@@ -287,7 +305,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
             }
           }
         }
-      } else if (MODE != kModeRowsum) {
+      } else if (!is_rowsum(MODE)) {
         // =============================================================== product MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1
         // Two issuing threads so that the per-tile bookkeeping of one overlaps the MMAs of the other.
         if (lane == 0) {
@@ -354,12 +372,108 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         const int row_in_tile = wq * 32 + lane;
         uint32_t gn0 = 0, n_grp = 0;
+        uint32_t ncol = 0;                             // symmetric row-sum mode: off-diagonal tiles this row tile has finished
         bool ok = true;
 
         for (int w = 0; w < my_items && ok; ++w) {
             FD_ITEM_GEOMETRY(w);
             const int64_t row = (int64_t)item * 256 + t * 128 + row_in_tile;
-            if (MODE == kModeRowsum) {
+            if constexpr (MODE == kModeRowsumSym) {
+                // Symmetric half-work row sums.  The S tile is built the other way round here (lanes = points of the
+                // STREAMED tile J, columns = points of the CTA's resident tile It), so a thread owns one streamed point:
+                //   * its sum over the 128 columns is that point's share of tile (J, It): one fixed-point atomic per tile;
+                //   * acc[c] += P[., c] collects, over the whole sweep, the resident point c's sum over the streamed
+                //     points that fall on this lane; the 128 lanes are reduced (butterfly of shuffles, the four warps
+                //     through shared memory) only every kSymFlush tiles, which also bounds the fp32 accumulation length.
+                // J < It is the mirror of a tile another resident tile evaluates (skipped: only J = 2 item for the second
+                // resident tile); J == It counts once (resident side only); J > It counts for both sides.  Sums go to one
+                // 64-bit fixed-point integer per point: integer additions commute, so the result does not depend on the
+                // order in which CTAs arrive.
+                constexpr int kSymFlush = 64;
+                float* colpart = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 1024);
+                const double fix = (double)(1ull << p.sym_shift);
+                const int It = 2 * item + t;
+                float acc[128];
+#pragma unroll
+                for (int c = 0; c < 128; ++c) acc[c] = 0.f;
+                double dsq = 0.0;
+                int pending = 0;                               // tiles accumulated in acc since the last reduction
+                // reduces acc over the 128 lanes of the resident tile and adds the sums to the resident points
+                auto reduce_acc = [&]() -> bool {
+                    const uint32_t slot = ncol & 1u;
+                    float* mine = colpart + (((t * 2 + (int)slot) * 4 + wq) * 128);
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+#pragma unroll
+                        for (int m = 16; m >= 1; m >>= 1) {
+                            const bool up = (lane & m) != 0;
+#pragma unroll
+                            for (int k = 0; k < m; ++k) {
+                                const float send = up ? acc[32 * ch + k] : acc[32 * ch + k + m];
+                                const float keep = up ? acc[32 * ch + k + m] : acc[32 * ch + k];
+                                acc[32 * ch + k] = keep + __shfl_xor_sync(0xffffffffu, send, m);
+                            }
+                        }
+                        mine[ch * 32 + lane] = acc[32 * ch];
+                    }
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) acc[c] = 0.f;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->col_ready[t][slot]);
+                    if (!mbar_wait(&bars->col_ready[t][slot], (ncol >> 1) & 1u, abort_flag, p.status, 11)) return false;
+                    const float* all = colpart + ((t * 2 + (int)slot) * 4) * 128;
+                    const int cidx = wq * 32 + lane;
+                    const float csum = (all[cidx] + all[128 + cidx]) + (all[256 + cidx] + all[384 + cidx]);
+                    const int64_t pt = (int64_t)It * 128 + cidx;
+                    if (pt < p.N) atomicAdd(p.symsum + pt, (unsigned long long)__double2ll_rn((double)csum * fix));
+                    ++ncol;
+                    return true;
+                };
+                for (int j = 0; j < num_jt && ok; ++j) {
+                    const uint32_t g = gn0 + 2u * j + t;
+                    const int buf = g % NBUF;
+                    ok = mbar_wait(&bars->s_full[buf][t], (g / kRingPeriod) & 1, abort_flag, p.status, 8);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t addr = tmem + lane_addr + 128u * buf;
+                    const int J = j0 + j;
+                    const bool use = J >= It;
+                    float r0 = 0.f, r1 = 0.f, q0 = 0.f, q1 = 0.f;
+                    uint32_t sv[2][32];
+                    tmem_ld32(addr, sv[0]);
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        tmem_wait_ld();
+                        if (ch < 3) tmem_ld32(addr + 32 * (ch + 1), sv[(ch + 1) & 1]);
+                        if (use) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const float p0 = ex2f(__uint_as_float(sv[ch & 1][i])), p1 = ex2f(__uint_as_float(sv[ch & 1][i + 1]));
+                                acc[32 * ch + i] += p0; acc[32 * ch + i + 1] += p1;
+                                r0 += p0; r1 += p1;
+                                q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1);
+                            }
+                        }
+                    }
+                    // the buffer can be refilled: its values are in registers or consumed
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->s_done[buf][t]);
+                    if (!use) continue;                            // mirrored tile: evaluated by the other resident tile
+                    const bool offdiag = J > It;
+                    dsq += (double)(q0 + q1) * (offdiag ? 2.0 : 1.0);
+                    if (offdiag) {
+                        const int64_t pt = (int64_t)J * 128 + row_in_tile;
+                        if (pt < p.N) atomicAdd(p.symsum + pt, (unsigned long long)__double2ll_rn((double)(r0 + r1) * fix));
+                    }
+                    if (++pending == kSymFlush) { ok = reduce_acc(); pending = 0; if (!ok) break; }
+                }
+                if (ok && pending > 0) ok = reduce_acc();
+                if (ok && num_jt > 0 && row < p.Nrow && p.rowsq)
+                    // this thread's share of sum_ij K_ij^2: only the total over all threads is meaningful.  (A thread whose
+                    // slot It * 128 + r lies beyond N has only seen streamed points J * 128 + r >= N, i.e. zeros.)
+                    p.rowsq[row] = dsq * (1.0 / ((double)(1 << kBias) * (double)(1 << kBias)));
+            } else if (MODE == kModeRowsum) {
                 double dsum = 0.0, dsq = 0.0;
                 for (int j = 0; j < num_jt && ok; ++j) {
                     const uint32_t g = gn0 + 2u * j + t;
@@ -514,7 +628,7 @@ __global__ void k_wait_selftest(unsigned int* status, long long limit_cycles) {
 
 // ------------------------------------------------------------------------------------------------ operand packing
 // Augmented fp16 hi|lo operand rows.  role 0 (rows of the product): [c x, e, 1]; role 1 (columns): [c x, 1, e] with
-// c = sqrt(2 b'), e = -b' |x - mu|^2 (+ extra_j: bias and log2 of a positive right vector for role 1).
+// c = sqrt(2 b'), e = -b' |x - mu|^2 (+ the bias for role 1, + log2 of a positive weight vector when one is given).
 // Layout: slab s (16 augmented columns) of point p at out[(s * np + p) * 32 ..]: 16 hi then 16 lo halves.
 __global__ void k_pack_points(const float* __restrict__ xs, int DP, int D, int64_t n, int64_t np, const double* __restrict__ mu,
                               double bprime, int role, double bias, const float* __restrict__ logw_src, int K16,
@@ -527,11 +641,9 @@ __global__ void k_pack_points(const float* __restrict__ xs, int DP, int D, int64
     if (valid)
         for (int k = 0; k < D; ++k) { double v = (double)xs[pidx * DP + k] - mu[k]; r += v * v; }
     double e = -bprime * r;
-    if (role == 1) {
-        e += bias;
-        if (logw_src && valid) e += log2((double)logw_src[pidx]);
-        if (!valid) e = -30000.0;                       // padded column: 2^e = 0
-    }
+    if (logw_src && valid) e += log2((double)logw_src[pidx]);     // a positive weight rides in the exponent
+    if (role == 1) e += bias;
+    if (!valid) e = -30000.0;                           // padded point: 2^e = 0 (its row / column contributes nothing)
     // norm pieces: two hi/lo pairs carry e to beyond fp32 precision
     const __half e_h1 = __double2half(e);
     const double r1 = e - (double)__half2float(e_h1);
@@ -552,7 +664,7 @@ __global__ void k_pack_points(const float* __restrict__ xs, int DP, int D, int64
                     l = __double2half(v - (double)__half2float(h));
                 }
             } else if (col == D || col == D + 1) {          // row-norm slots: role 0 carries e, role 1 carries 1
-                if (role == 0) { h = col == D ? e_h1 : e_h2; l = col == D ? e_l1 : e_l2; if (!valid) { h = zero; l = zero; } }
+                if (role == 0) { h = col == D ? e_h1 : e_h2; l = col == D ? e_l1 : e_l2; }
                 else h = one;
             } else if (col == D + 2 || col == D + 3) {      // column-norm slots
                 if (role == 1) { h = col == D + 2 ? e_h1 : e_h2; l = col == D + 2 ? e_l1 : e_l2; }
@@ -618,6 +730,12 @@ __global__ void k_pack_wt(const float* __restrict__ V, int64_t ldv, const float*
         hi[(int64_t)c * np + j] = h;
         if (lo) lo[(int64_t)c * np + j] = __float2half_rn(v - __half2float(h));
     }
+}
+
+// Symmetric row-sum mode: fixed-point sums -> q.
+__global__ void k_sym_finish(const unsigned long long* __restrict__ sums, int64_t n, double scale, float* __restrict__ q) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) q[i] = (float)((double)(long long)sums[i] * scale);
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -702,7 +820,12 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(c->xs(), L.DP, L.D, N, NP, mu, bprime, 1, (double)kBias,
                                                    rowsum ? a.right : nullptr, K16, xp_col);
     FD_LAUNCH_CHECK(c, "k_pack_points(col)");
-    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(a.xrow, L.DP, L.D, a.Nrow, NP, mu, bprime, 0, 0.0, nullptr, K16, xp_row);
+    // Symmetric row sums (K = K^T): a square pass over the context's own points whose left and right weights are the same
+    // vector (the degree passes) evaluates only the tiles on or above the diagonal; the weight is folded into both exponents.
+    const bool sym = rowsum && a.sym_ok && c->opt_sym != 0 && a.rows_are_ctx && a.xrow == c->xs() && a.Nrow == N &&
+                     a.left == a.right && L.symsum != 0;
+    k_pack_points<<<pk_blocks, 256, 0, c->stream>>>(a.xrow, L.DP, L.D, a.Nrow, NP, mu, bprime, 0, 0.0, sym ? a.right : nullptr, K16,
+                                                   xp_row);
     FD_LAUNCH_CHECK(c, "k_pack_points(row)");
 
     CUtensorMap mr, mc, mh, ml;
@@ -723,7 +846,22 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
     p.flush = c->opt_flush > 0 ? c->opt_flush : 1;
     const int grid = std::min(p.num_work, c->sm_count);
 
-    if (rowsum) {
+    if (rowsum && sym) {
+        p.num_jt = (int)(NP / 128);                      // even: every row pair's two diagonal tiles exist (padding gives 2^e = 0)
+        p.jt_chunk = p.num_jt; p.num_chunks = 1;
+        p.left = nullptr;
+        p.q = a.Y; p.rowsq = a.rowsq; p.b = 1;
+        p.symsum = c->at<unsigned long long>(L.symsum);
+        // sums are at most NP * 2^bias in the kernel's scaled units: the fixed-point unit keeps them below 2^61
+        int lg = 0;
+        while (((int64_t)1 << lg) < NP) ++lg;
+        p.sym_shift = 61 - kBias - lg;
+        FD_CUDA(c, cudaMemsetAsync(p.symsum, 0, (size_t)N * 8, c->stream));
+        const int sym_grid = std::min((p.num_work + 1) / 2, c->sm_count);
+        FD_TRY((launch_tc<16, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
+        k_sym_finish<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(p.symsum, N, std::ldexp(1.0, -(kBias + p.sym_shift)), a.Y);
+        FD_LAUNCH_CHECK(c, "k_sym_finish");
+    } else if (rowsum) {
         p.q = a.Y; p.rowsq = a.rowsq; p.b = 1;
         FD_TRY((launch_tc<16, kModeRowsum>(c, mr, mc, mc, mc, p, grid)));
     } else {

@@ -14,7 +14,10 @@ constexpr int kBias = 15;                    // P' = 2^15 P keeps fp16 hi/lo of 
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any legitimate wait
 
-enum Mode { kModeBlock = 0, kModeRowsum = 2 };
+// kModeRowsumSym: row sums of a SYMMETRIC weighted kernel matrix from its upper triangle of tiles alone (K = K^T, Sec.
+// 2.1): every off-diagonal tile also yields the column sums that the mirrored tile's rows would have computed.
+enum Mode { kModeBlock = 0, kModeRowsum = 2, kModeRowsumSym = 3 };
+__host__ __device__ constexpr bool is_rowsum(int mode) { return mode == kModeRowsum || mode == kModeRowsumSym; }
 
 struct TcParams {
     int64_t Nrow, N;             // valid rows / columns
@@ -30,6 +33,8 @@ struct TcParams {
     const float* colscale_inv;   // per column: 2^-bias / colscale
     float* Y; int64_t ldy;
     float* q; double* rowsq;     // row-sum outputs
+    unsigned long long* symsum;  // symmetric row-sum mode: fixed-point row + column sums, one 64-bit integer per point
+    int sym_shift;               // ... in units of 2^-sym_shift of the (2^bias-scaled) kernel values
     unsigned int* status;
 };
 

@@ -110,6 +110,44 @@ def test_non_finite_points_are_refused(fd, dev):
     assert e.value.status == fd.FD_ERR_NONFINITE
 
 
+@pytest.mark.parametrize("N", [1, 100, 256, 257, 600, 1000, 2304, 5000])
+@pytest.mark.parametrize("alpha", [0.0, 1.0])
+def test_symmetric_half_work_degree_passes(fd, dev, N, alpha):
+    """K = K^T (Sec. 2.1): the degree passes evaluate only the tiles on or above the diagonal and take the mirrored half
+    from column sums.  Same gates against the oracle as the full evaluation, agreement with it to fp32 rounding, identical
+    bits from run to run (fixed-point sums), odd and even numbers of row pairs, padding inside the last tiles."""
+    X = workloads.torus6(N, seed=N + 7)
+    beta = 2.0
+    ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=8)
+    ctx.set_option("path", fd.FD_PATH_TC)
+    out = {}
+    for sym in (1, 0, 1):
+        ctx.set_option("sym", sym)
+        q, d, s, so, so2 = ctx.degree(beta, alpha)
+        assert ctx.get_option("last_path") == fd.FD_PATH_TC
+        res = (q.cpu().numpy(), d.cpu().numpy(), s.cpu().numpy(), so, so2)
+        if sym == 1 and 1 in out:
+            for a, b in zip(res[:3], out[1][:3]):
+                assert np.array_equal(a, b)
+            assert res[3:] == out[1][3:]
+        out[sym] = res
+    qo, do, s_o, soo, so2o = dense.degree(X, beta, alpha)
+    for sym in (1, 0):
+        q, d, s, so, so2 = out[sym]
+        assert np.abs(q / qo - 1).max() <= TOL_DEG
+        assert np.abs(d / do - 1).max() <= 2 * TOL_DEG and np.abs(s / s_o - 1).max() <= 2 * TOL_DEG
+        assert abs(so - soo) <= TOL_DEG * (soo + N) and abs(so2 - so2o) <= 2 * TOL_DEG * (so2o + N)
+    assert np.abs(out[1][0] / out[0][0] - 1).max() <= 2e-6 and np.abs(out[1][1] / out[0][1] - 1).max() <= 4e-6
+    # the block product with the half-work scale vector
+    V = workloads.block(N, 8 if N > 1 else 1, seed=2)
+    ctx.set_option("sym", 1)
+    ctx.degree(beta, alpha)
+    Y = ctx.apply(fd.to_colmajor(V, dev))
+    ctx.synchronize()
+    assert relF(Y.cpu().numpy(), dense.apply(X, beta, alpha, V)) <= TOL_APPLY
+    ctx.close()
+
+
 @pytest.mark.parametrize("alpha", [0.0, 0.5, 1.0])
 def test_alpha(fd, dev, alpha):
     tc_case(fd, dev, workloads.torus6(1500, seed=4), 1.5, alpha, 32)
