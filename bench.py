@@ -380,14 +380,22 @@ def run_gpu(args):
                                                  "product_24_mma_ts_n64": 24 * rates["clk_mma_ts_n64"],
                                                  "mufu_128x128_exps": 128 * 128 / rates["ex2_per_clk_sm"]},
                     "unit_rates": rates}
-        deg_pairs_per_s = 2.0 * units / b / (deg_ms * 1e-3)       # per GPU
+        deg_pairs_per_s = 2.0 * units / b / (deg_ms * 1e-3)       # per GPU: pairs SERVED per second (both passes)
+        # exponentials the two passes actually execute: all N^2 per pass, or -- on the Gram-form kernels of an unsharded
+        # context, which use K = K^T -- only the 128 x 128 tiles on or above the diagonal: T (T + 1) / 2 tiles, T = ceil(N / 256) * 2
+        sym_on = path_used == "tc" and not sharded and ctx.get_option("sym") == 1
+        T = -(-N // 256) * 2
+        deg_exps = 2.0 * (T * (T + 1) // 2 * 16384 if sym_on else float(N) * N / (world if sharded else 1))
         out = {"metric": METRIC, "value": job_value(units, world, app_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
                "apply_ms": app_ms, "path": path_used, "roofline": roofline,
                "whole_step": {"ms": step_ms, "pair_cols_per_s": job_value(units * (b + 2) / b, world, step_ms),
                               "note": "degree pass + second normalisation pass + scale vector + block product"},
-               "degree_passes": {"ms_both": deg_ms, "pairs_per_s": deg_pairs_per_s, "frac_of_mufu_peak": deg_pairs_per_s / mufu_peak},
+               "degree_passes": {"ms_both": deg_ms, "pairs_served_per_s": deg_pairs_per_s, "symmetric_half_work": bool(sym_on),
+                                 "executed_exponentials_both_passes": deg_exps,
+                                 "frac_of_mufu_peak": deg_exps / (deg_ms * 1e-3) / mufu_peak,
+                                 "note": "frac counts the exponentials actually executed (never the pairs served), against the same MUFU peak"},
                "fast_mode_apply": None if fast_ms is None else {
                    "ms": fast_ms, "pair_cols_per_s": units / (fast_ms * 1e-3), "frac_of_mufu_peak": units / b / (fast_ms * 1e-3) / mufu_peak,
                    "note": "FD_PREC_FAST: single fp16 operands, relative Frobenius error ~2e-4 (bound 3e-3); reported separately"},
