@@ -871,8 +871,12 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
         float* inv = scale + L.BP + 8;
         float* part = c->at<float>(L.part);
         const bool fast = a.prec == FD_PREC_FAST;
-        for (int c0 = 0; c0 < a.b; c0 += 64) {
-            const int bc = std::min(64, a.b - c0);
+        // widest column chunk whose stages fit in shared memory: 64 columns up to D = 28, 32 up to D = 44, 16 beyond (the
+        // fp32-grade kernel stages W_hi and W_lo; the reduced-precision kernel stages one of them and always fits 64)
+        const int limit = 227 * 1024;
+        const int cw = fast || Smem<64, kModeBlock>::total(K16) <= limit ? 64 : Smem<32, kModeBlock>::total(K16) <= limit ? 32 : 16;
+        for (int c0 = 0; c0 < a.b; c0 += cw) {
+            const int bc = std::min(cw, a.b - c0);
             const int BT = bc <= 16 ? 16 : bc <= 32 ? 32 : 64;
             if (BT > L.BP) return fail(c, FD_ERR_WORKSPACE, "column tile %d wider than the provisioned block buffers (%d)", BT, L.BP);
             const int cm_blocks = (int)std::min<int64_t>(256, ceil_div(N, 1024));

@@ -78,6 +78,17 @@ def test_dimensions_and_k_slabs(fd, dev, D, beta):
     tc_case(fd, dev, X, beta, 1.0, 32)
 
 
+@pytest.mark.parametrize("D,b", [(30, 64), (32, 48), (40, 64), (50, 40), (60, 64)])
+def test_wide_blocks_at_large_dimension_are_served_in_narrower_chunks(fd, dev, D, b):
+    # the stages of a 64-column chunk do not fit in shared memory beyond D = 28 (fp32-grade kernel): the product is then
+    # swept in 32- or 16-column chunks; the reduced-precision kernel keeps 64
+    X = workloads.latent_torus(1500, seed=D, D=D)
+    beta = 0.3
+    err = tc_case(fd, dev, X, beta, 1.0, b)
+    assert err <= TOL_APPLY
+    tc_case(fd, dev, X, beta, 1.0, b, prec=1)
+
+
 def test_dimensions_33_to_60_take_the_gram_form_path_at_any_size(fd, dev):
     # 32 < D <= 60 is covered by the tensor-core family alone: the automatic choice must pick it even for a small point
     # set, and a bandwidth beyond its accuracy budget is refused instead of silently served by nothing
