@@ -390,6 +390,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 // 64-bit fixed-point integer per point: integer additions commute, so the result does not depend on the
                 // order in which CTAs arrive.
                 constexpr int kSymFlush = 64;
+                constexpr bool kWantSq = BT == 16;             // the sum of squares rides along in the first degree pass only (BT = 32: without)
                 float* colpart = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 1024);
                 const double fix = (double)(1ull << p.sym_shift);
                 const int It = 2 * item + t;
@@ -451,7 +452,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                                 const float p0 = ex2f(__uint_as_float(sv[ch & 1][i])), p1 = ex2f(__uint_as_float(sv[ch & 1][i + 1]));
                                 acc[32 * ch + i] += p0; acc[32 * ch + i + 1] += p1;
                                 r0 += p0; r1 += p1;
-                                q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1);
+                                if (kWantSq) { q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1); }
                             }
                         }
                     }
@@ -858,7 +859,8 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
         p.sym_shift = 61 - kBias - lg;
         FD_CUDA(c, cudaMemsetAsync(p.symsum, 0, (size_t)N * 8, c->stream));
         const int sym_grid = std::min((p.num_work + 1) / 2, c->sm_count);
-        FD_TRY((launch_tc<16, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
+        if (p.rowsq) FD_TRY((launch_tc<16, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
+        else FD_TRY((launch_tc<32, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
         k_sym_finish<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(p.symsum, N, std::ldexp(1.0, -(kBias + p.sym_shift)), a.Y);
         FD_LAUNCH_CHECK(c, "k_sym_finish");
     } else if (rowsum) {
