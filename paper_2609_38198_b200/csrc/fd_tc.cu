@@ -499,7 +499,9 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                             const float p0 = ex2f(__uint_as_float(sv[ch][i])), p1 = ex2f(__uint_as_float(sv[ch][i + 1]));
                             const float p2 = ex2f(__uint_as_float(sv[ch][i + 2])), p3 = ex2f(__uint_as_float(sv[ch][i + 3]));
                             a0 += p0; a1 += p1; a2 += p2; a3 += p3;
-                            q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1); q0 = fmaf(p2, p2, q0); q1 = fmaf(p3, p3, q1);
+                            if (BT == 16) {                // (BT = 32: the instantiation without the sum of squares)
+                                q0 = fmaf(p0, p0, q0); q1 = fmaf(p1, p1, q1); q0 = fmaf(p2, p2, q0); q1 = fmaf(p3, p3, q1);
+                            }
                         }
                     }
                     dsum += (double)((a0 + a1) + (a2 + a3));
@@ -865,7 +867,8 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
         FD_LAUNCH_CHECK(c, "k_sym_finish");
     } else if (rowsum) {
         p.q = a.Y; p.rowsq = a.rowsq; p.b = 1;
-        FD_TRY((launch_tc<16, kModeRowsum>(c, mr, mc, mc, mc, p, grid)));
+        if (p.rowsq) FD_TRY((launch_tc<16, kModeRowsum>(c, mr, mc, mc, mc, p, grid)));
+        else FD_TRY((launch_tc<32, kModeRowsum>(c, mr, mc, mc, mc, p, grid)));
     } else {
         __half* wt_hi = c->at<__half>(L.wt_hi);
         __half* wt_lo = c->at<__half>(L.wt_lo);
