@@ -190,3 +190,45 @@ def test_exchange_failure_is_reported_not_hung(fd, dev):
     q = ctx.degree(1.0, 1.0)[0].cpu().numpy()
     assert np.abs(q / dense.degree(X, 1.0, 1.0)[0] - 1).max() <= 2e-5
     ctx.close()
+
+
+def test_torch_distributed_transport_on_a_one_rank_group(fd, dev):
+    """The transport a multi-GPU job uses -- NCCL all_gather_into_tensor on the context's stream for the row gathers, a gloo
+    group for the small host sums -- on a one-rank group, which needs only this GPU: degree passes, block product and
+    eigensolver through fd_set_shard against the oracle."""
+    import socket
+
+    import torch.distributed as dist
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        host_group = dist.new_group(backend="gloo")
+        N, b, beta, alpha, k = 3000, 16, 1.0, 1.0, 6
+        X = workloads.torus6(N, seed=77)
+        V = workloads.block(N, b, seed=5)
+        for path in (fd.FD_PATH_SIMT, fd.FD_PATH_TC):
+            ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=64)
+            ctx.set_option("path", path)
+            ctx.set_shard(fd.Shard(fd.TorchDistTransport(0, 1, group=None, host_group=host_group), N, b, dev))
+            q, d, s, so, so2 = ctx.degree(beta, alpha)
+            Y = ctx.apply(fd.to_colmajor(V, dev))
+            lam, U, info = ctx.eigs(k, 8)
+            ctx.synchronize()
+            qo, do, s_o, soo, so2o = dense.degree(X, beta, alpha)
+            assert np.abs(q.cpu().numpy() / qo - 1).max() <= 2e-5 and abs(so - soo) <= 2e-5 * (soo + N)
+            assert relF(Y.cpu().numpy(), dense.apply(X, beta, alpha, V)) <= TOL_APPLY
+            lam_o, U_o, d_o = dense.eigs(X, beta, alpha, k)
+            assert info.converged == k + 1 and np.abs(lam - lam_o).max() <= 1e-6
+            ctx.close()
+        # without a host group the small sums are staged through the device on the NCCL group
+        ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b, m_max=64)
+        ctx.set_shard(fd.Shard(fd.TorchDistTransport(0, 1, group=None, host_group=None), N, b, dev))
+        q2 = ctx.degree(beta, alpha)[0]
+        assert np.abs(q2.cpu().numpy() / qo - 1).max() <= 2e-5
+        ctx.close()
+    finally:
+        dist.destroy_process_group()
