@@ -405,6 +405,8 @@ def run_gpu(args):
                        "note": "host buffers: H2D of X and V, fd_create, degree passes, block product, D2H of Y",
                        "h2d_bytes_per_step": int(Xh.numel() * 4 + Vh.numel() * 4), "d2h_bytes_per_step": int(Yh.numel() * 4)},
                "gpu_launches": int(launches), "workspace_bytes": ctx.workspace_bytes}
+        if world == 1 and not sharded:
+            out["sharded_rank_share"] = sharded_rank_share(fd, dev, Xd, Vd, Yd, beta, alpha, b)
         if not args.no_cpu and world == 1:
             out["cpu_baseline"] = cpu_baseline(X, V, cfg)
     ctx.close()
@@ -579,6 +581,46 @@ def paper_shape_context(fd, dev):
             out.append({"N": N, "D": 32, "beta": 1.0, "b": b, "seconds": t, "pair_cols_per_s": float(N) * N * b / t,
                         "path": "tc" if ctx.get_option("last_path") == 2 else "simt",
                         "printed_seconds_other_gpu": printed[(N, b)]})
+        ctx.close()
+    return out
+
+
+def sharded_rank_share(fd, dev, Xd, Vd, Yd, beta, alpha, b):
+    """What ONE rank of a row-sharded job computes, measured on this GPU with the exchange stubbed out (a transport whose
+    gathers and sums do nothing): the block product and the degree passes over rank 0's rows of a 2-, 4- and 8-rank
+    partition, pack / unpack copies of the gather included, the NCCL transfer itself (N b 4 bytes per product over
+    NVLink) not.  The figures say how the work divides; they are not a multi-GPU measurement."""
+    import torch
+    N = Xd.shape[0]
+
+    class Stub:
+        def __init__(self, world):
+            self.rank, self.world = 0, world
+
+        def allreduce_sum_host(self, arr, device, stream):
+            pass
+
+        def allgather(self, send, recv, stream):
+            pass
+
+    out = []
+    for world in (2, 4, 8):
+        ctx = fd.Context(Xd, b_max=b, m_max=0)
+        ctx.set_shard(fd.Shard(Stub(world), N, b, dev))
+        ctx.degree(beta, alpha)
+        ctx.apply(Vd, out=Yd)
+        torch.cuda.synchronize(dev)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        ctx.degree(beta, alpha)
+        e[1].record()
+        for _ in range(3):
+            ctx.apply(Vd, out=Yd)
+        e[2].record()
+        torch.cuda.synchronize(dev)
+        r0, r1 = fd.fd_shard_rows(N, world, 0)
+        out.append({"world": world, "rows_of_rank_0": r1 - r0, "apply_ms": e[1].elapsed_time(e[2]) / 3.0,
+                    "degree_passes_ms": e[0].elapsed_time(e[1]), "gather_bytes_per_apply": int(N) * b * 4})
         ctx.close()
     return out
 
