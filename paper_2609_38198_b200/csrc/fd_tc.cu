@@ -15,8 +15,12 @@
 //      so tensor-core accumulation error does not grow with N.
 // S tiles flow through a ring of TMEM buffers shared by both row tiles, so the tensor core runs ahead of
 // the warpgroups and the product MMA of a tile overlaps the exponentials of the next ones.
-// Row-sum mode (degree passes): no product MMA; the warpgroups add P (and P^2) on the FMA pipe,
+// Row-sum mode (rectangular and row-sharded passes): no product MMA; the warpgroups add P (and P^2) on the FMA pipe,
 // fp32 within a column tile and fp64 across tiles; a positive right vector enters through e_j.
+// Symmetric row-sum mode (the degree passes of a whole data set, K = K^T): only the tiles on or above the diagonal are
+// evaluated; the S tile is built with the streamed points on the TMEM lanes, so one thread adds up both what a tile gives
+// its streamed point (one fixed-point atomic per tile) and, in 128 per-thread accumulators reduced across lanes every
+// 64 tiles, what it gives the resident points.
 //
 // One persistent CTA per SM: warps 0-3 / 4-7 = the two exponential warpgroups (raised to 232 registers);
 // warp 8 = TMA producer, warps 9 / 10 = product-MMA issuers for row tile 0 / 1, warp 11 = Gram-MMA issuer
