@@ -200,6 +200,10 @@ def spawn_ranks(args) -> int:
 
 # ------------------------------------------------------------------------------------------- GPU arm
 def run_gpu(args):
+    # stdout carries the one JSON line: NCCL prints a version banner there at NCCL_DEBUG=VERSION (and at WARN), so that
+    # setting is dropped; the library reads the variable once, so this has to happen before torch loads it
+    if os.environ.get("NCCL_DEBUG", "").upper() == "VERSION":
+        del os.environ["NCCL_DEBUG"]
     import torch
     import __graft_entry__ as entry
     entry.build()
