@@ -235,3 +235,40 @@ def test_beta0_matches_oracle(fd, dev):
         ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=1)
         assert ctx.beta0() == pytest.approx(flow.beta0(X), rel=1e-6)
         ctx.close()
+
+
+# ------------------------------------------------------------------ seeded sweep over shapes, both kernel families
+@pytest.mark.parametrize("seed", range(20))
+def test_seeded_shape_sweep_both_families(fd, dev, seed):
+    """Random (N, D, b, alpha, beta) drawn from a seed: ragged sizes around the tile edges, every dimension the kernels
+    cover, block widths that straddle the column-tile widths.  Each shape runs on every kernel family that covers it
+    (direct differences for D <= 32, Gram form for D <= 60 within its accuracy budget), against the dense oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    N = int(rng.choice([1, 2, 31, 127, 128, 129, 255, 256, 257, 383, 511, 640, 1000, 1537, 2049, 2600]))
+    D = int(rng.integers(1, 61))
+    b = int(rng.choice([1, 2, 7, 8, 15, 16, 17, 31, 32, 33, 47, 63, 64, 65, 100]))
+    alpha = float(rng.choice([0.0, 0.5, 1.0]))
+    X = workloads.gaussian_cloud(N, D, seed=seed, scale=0.6)
+    # bandwidth: a few tens of effective neighbours, and an exponent magnitude the Gram form is trusted with
+    mu = X.mean(axis=0, keepdims=True)
+    max_sq = float(((X - mu) ** 2).sum(axis=1).max()) if N > 1 else 1.0
+    beta = float(min(2.0 / (0.36 * D), 40.0 / (1.4427 * max(max_sq, 1e-3))))
+    V = workloads.block(N, b, seed=seed + 5)
+    qo, do, s_o, soo, so2o = dense.degree(X, beta, alpha)
+    Yo = dense.apply(X, beta, alpha, V)
+    paths = ([fd.FD_PATH_SIMT] if D <= 32 else []) + [fd.FD_PATH_TC]
+    for path in paths:
+        tol = 1e-5 if path == fd.FD_PATH_SIMT else 2e-5
+        ctx = fd.Context(torch.from_numpy(X).to(dev), b_max=b)
+        ctx.set_option("path", path)
+        q, d, s, so, so2 = ctx.degree(beta, alpha)
+        Y = ctx.apply(fd.to_colmajor(V, dev)) if N > 1 or b == 1 else None
+        ctx.synchronize()
+        assert ctx.get_option("last_path") == path
+        assert np.abs(q.cpu().numpy() / qo - 1).max() <= tol, (N, D, b, path)
+        assert np.abs(d.cpu().numpy() / do - 1).max() <= 2 * tol and np.abs(s.cpu().numpy() / s_o - 1).max() <= 2 * tol
+        assert abs(so - soo) <= tol * (soo + N) and abs(so2 - so2o) <= 2 * tol * (so2o + N)
+        if Y is not None:
+            err = relF(Y.cpu().numpy(), Yo)
+            assert err <= TOL_APPLY, (N, D, b, alpha, beta, path, err)
+        ctx.close()
