@@ -91,7 +91,10 @@ fd_status fd_destroy(fd_ctx* ctx);
  * tiles per L2-resident chunk of the tensor-core block product), "sym" (1, default: the degree passes on the Gram-form
  * kernels use K = K^T and evaluate only the tiles on or above the diagonal -- each off-diagonal tile gives the row sums
  * of its rows and, transposed, of its columns, N (N + 128) / 2 exponentials instead of N^2; 0: every tile; row-sharded
- * contexts always evaluate every tile of their rows), "wait_selftest" (value = limit in SM cycles: enqueues
+ * contexts always evaluate every tile of their rows), "tail_split" (1, default: in a block product with a single column
+ * chunk the row pairs of the last, partly filled round of CTAs -- all pairs when there are fewer than CTAs -- are
+ * shared by two CTAs each, half the columns per CTA, partial results added atomically; 0: off), "wait_selftest"
+ * (value = limit in SM cycles: enqueues
  * a one-thread kernel whose bounded wait on a barrier that nothing completes must expire; the next
  * fd_synchronize then returns FD_ERR_TIMEOUT and the context stays usable).  fd_get_option also reports "last_path" (the
  * family that served the latest pass), "beta", "mean_sq", "max_sq" and "tc_cycles" (SM cycles the first CTA of the most

@@ -156,6 +156,9 @@ fd_status fd_set_option(fd_ctx* c, const char* name, double v) {
     } else if (!strcmp(name, "flush")) {
         if (v < 0 || v > 1 << 20) return fail(c, FD_ERR_INVALID, "flush out of range");
         c->opt_flush = (int)v;
+    } else if (!strcmp(name, "tail_split")) {
+        if (v != 0 && v != 1) return fail(c, FD_ERR_INVALID, "tail_split must be 0 or 1");
+        c->opt_tail_split = (int)v;
     } else if (!strcmp(name, "sym")) {
         if (v != 0 && v != 1) return fail(c, FD_ERR_INVALID, "sym must be 0 or 1");
         c->opt_sym = (int)v;
@@ -180,6 +183,7 @@ fd_status fd_get_option(const fd_ctx* c, const char* name, double* v) {
     else if (!strcmp(name, "splits")) *v = c->opt_splits;
     else if (!strcmp(name, "flush")) *v = c->opt_flush;
     else if (!strcmp(name, "sym")) *v = c->opt_sym;
+    else if (!strcmp(name, "tail_split")) *v = c->opt_tail_split;
     else if (!strcmp(name, "tc_max_mag")) *v = c->opt_tc_max_mag;
     else if (!strcmp(name, "last_path")) *v = c->last_path;
     else if (!strcmp(name, "tc_cycles")) {

@@ -56,6 +56,7 @@ struct fd_ctx {
     int opt_path = FD_PATH_AUTO;
     int opt_splits = 0;
     int opt_flush = 0;
+    int opt_tail_split = 1;          // block product, single column chunk: share the last round's row pairs between two CTAs each
     int opt_sym = 1;                 // symmetric half-work degree passes on the Gram-form kernels (0 = evaluate every tile)
     int opt_jt_chunk = 0;            // column tiles per L2-resident chunk of the tensor-core block product (0 = default)
     int last_path = 0;               // kernel family that served the most recent quadratic pass (FD_PATH_SIMT / FD_PATH_TC)

@@ -130,17 +130,26 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     // item is empty).
     constexpr bool kSym = MODE == kModeRowsumSym;
     const int sym_units = (p.num_work + 1) / 2;
+    const bool kTail = !kSym && p.tail_split == 2;
+    const int full_rounds = kTail ? p.tail_first / (int)gridDim.x : 0;
     const int my_rows = kSym ? (sym_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
                              : (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_items = kSym ? 2 * my_rows : my_rows * p.num_chunks;
+    const int my_items = kSym ? 2 * my_rows
+                       : kTail ? full_rounds + ((int)blockIdx.x < 2 * p.tail_pairs ? 1 : 0) : my_rows * p.num_chunks;
+    const int tail_half = (p.num_jt + 1) / 2;
 #define FD_ITEM_GEOMETRY(w)                                                                         \
-    const int unit_ = (int)blockIdx.x + (kSym ? ((w) >> 1) : ((w) % my_rows)) * (int)gridDim.x;     \
-    const int cch = kSym ? 0 : (w) / my_rows;                                                       \
-    const int item = (kSym && ((w) & 1)) ? p.num_work - 1 - unit_ : unit_;                          \
-    const int j0 = kSym ? 2 * item : cch * p.jt_chunk;                                              \
+    const bool tail_item = kTail && (w) >= full_rounds;                                             \
+    const int tail_part = tail_item ? (int)blockIdx.x / p.tail_pairs : 0;                           \
+    const int unit_ = (int)blockIdx.x + (kSym ? ((w) >> 1) : kTail ? (w) : ((w) % my_rows)) * (int)gridDim.x;     \
+    const int cch = (kSym || kTail) ? 0 : (w) / my_rows;                                            \
+    const int item = tail_item ? p.tail_first + (int)blockIdx.x % p.tail_pairs                      \
+                               : (kSym && ((w) & 1)) ? p.num_work - 1 - unit_ : unit_;              \
+    const int j0 = kSym ? 2 * item : tail_item ? tail_part * tail_half : cch * p.jt_chunk;          \
     const int num_jt = kSym ? ((((w) & 1) && item == unit_) ? 0 : p.num_jt - j0)                    \
+                     : tail_item ? (tail_part == 0 ? tail_half : p.num_jt - tail_half)              \
                             : ((p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk);          \
     const int tiles_per_item = 2 * num_jt;                                                          \
+    (void)tail_item; (void)tail_part;                                                               \
     (void)item; (void)tiles_per_item; (void)cch
     const int flush = p.flush;
 
@@ -604,7 +613,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         if (c < p.b) {
                             float* o = p.Y + row + (int64_t)c * p.ldy;
                             const float v = acc[c] * l * p.colscale_inv[c];
-                            *o = cch == 0 ? v : *o + v;          // later column chunks add to the partial result of the same thread
+                            if (tail_item) atomicAdd(o, v);      // the other half of the column range arrives from another CTA
+                            else *o = cch == 0 ? v : *o + v;     // later column chunks add to the partial result of the same thread
                         }
                 }
             }
@@ -907,10 +917,26 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
                 FD_TRY(launch_fast_product(c, BT, mr, mc, mh, pb, std::min(pb.num_work, c->sm_count)));
                 continue;
             }
+            // Tail split: with a single column chunk (N up to about 2^17) the row pairs of the last, partly filled round --
+            // or all pairs when there are fewer than CTAs -- are each shared by two CTAs (half the column range each).
+            int bgrid = grid;
+            p.tail_split = 0;
+            if (p.num_chunks == 1 && p.num_jt >= 2 && c->opt_tail_split != 0) {
+                const int tail = p.num_work % grid;                  // pairs in the last round (grid = min(pairs, SMs))
+                const int tail_pairs = p.num_work < c->sm_count ? p.num_work : tail;
+                if (tail_pairs > 0 && 2 * tail_pairs <= c->sm_count) {
+                    p.tail_split = 2;
+                    p.tail_pairs = tail_pairs;
+                    p.tail_first = p.num_work - tail_pairs;
+                    bgrid = std::max(grid, 2 * tail_pairs);
+                    const int64_t r0t = (int64_t)p.tail_first * 256;
+                    FD_CUDA(c, cudaMemset2DAsync(p.Y + r0t, (size_t)p.ldy * 4, 0, (size_t)(a.Nrow - r0t) * 4, (size_t)bc, c->stream));
+                }
+            }
             switch (BT) {
-                case 16: FD_TRY((launch_tc<16, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
-                case 32: FD_TRY((launch_tc<32, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
-                default: FD_TRY((launch_tc<64, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+                case 16: FD_TRY((launch_tc<16, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
+                case 32: FD_TRY((launch_tc<32, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
+                default: FD_TRY((launch_tc<64, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
             }
         }
     }

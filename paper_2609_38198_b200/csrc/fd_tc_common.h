@@ -24,6 +24,12 @@ struct TcParams {
     int num_work;                // row-pair tiles (256 rows each)
     int num_jt;                  // column tiles
     int jt_chunk, num_chunks;    // the column range is swept in chunks small enough for L2 (block mode); all CTAs work on one chunk at a time
+    // Tail split (block mode with a single column chunk): the row pairs left over after the full rounds -- all of them when
+    // there are fewer pairs than CTAs -- are each served by TWO CTAs, one per half of the column range, whose partial
+    // results meet in Y by atomic addition (Y zeroed beforehand; a sum of two terms does not depend on their order).
+    int tail_split;              // 0 = off, 2 = on
+    int tail_first;              // first row pair of the tail
+    int tail_pairs;              // number of row pairs in the tail
     int64_t np_rows;             // padded row count of the operand arrays (row index of K slab c = c * np + p)
     int64_t np_cols;
     int K16;
