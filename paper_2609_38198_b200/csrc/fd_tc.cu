@@ -130,7 +130,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     // item is empty).
     constexpr bool kSym = MODE == kModeRowsumSym;
     const int sym_units = (p.num_work + 1) / 2;
-    const bool kTail = !kSym && p.tail_split == 2;
+    constexpr bool kTail = MODE == kModeBlockTail;
     const int full_rounds = kTail ? p.tail_first / (int)gridDim.x : 0;
     const int my_rows = kSym ? (sym_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
                              : (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -613,8 +613,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                         if (c < p.b) {
                             float* o = p.Y + row + (int64_t)c * p.ldy;
                             const float v = acc[c] * l * p.colscale_inv[c];
-                            if (tail_item) atomicAdd(o, v);      // the other half of the column range arrives from another CTA
-                            else *o = cch == 0 ? v : *o + v;     // later column chunks add to the partial result of the same thread
+                            if (kTail && tail_item) atomicAdd(o, v);   // the other half of the column range arrives from another CTA
+                            else *o = cch == 0 ? v : *o + v;           // later column chunks add to the partial result of the same thread
                         }
                 }
             }
@@ -933,10 +933,18 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
                     FD_CUDA(c, cudaMemset2DAsync(p.Y + r0t, (size_t)p.ldy * 4, 0, (size_t)(a.Nrow - r0t) * 4, (size_t)bc, c->stream));
                 }
             }
+            if (p.tail_split == 2) {
+                switch (BT) {
+                    case 16: FD_TRY((launch_tc<16, kModeBlockTail>(c, mr, mc, mh, ml, p, bgrid))); break;
+                    case 32: FD_TRY((launch_tc<32, kModeBlockTail>(c, mr, mc, mh, ml, p, bgrid))); break;
+                    default: FD_TRY((launch_tc<64, kModeBlockTail>(c, mr, mc, mh, ml, p, bgrid))); break;
+                }
+                continue;
+            }
             switch (BT) {
-                case 16: FD_TRY((launch_tc<16, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
-                case 32: FD_TRY((launch_tc<32, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
-                default: FD_TRY((launch_tc<64, kModeBlock>(c, mr, mc, mh, ml, p, bgrid))); break;
+                case 16: FD_TRY((launch_tc<16, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+                case 32: FD_TRY((launch_tc<32, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
+                default: FD_TRY((launch_tc<64, kModeBlock>(c, mr, mc, mh, ml, p, grid))); break;
             }
         }
     }

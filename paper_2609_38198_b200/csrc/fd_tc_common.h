@@ -16,7 +16,9 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any legiti
 
 // kModeRowsumSym: row sums of a SYMMETRIC weighted kernel matrix from its upper triangle of tiles alone (K = K^T, Sec.
 // 2.1): every off-diagonal tile also yields the column sums that the mirrored tile's rows would have computed.
-enum Mode { kModeBlock = 0, kModeRowsum = 2, kModeRowsumSym = 3 };
+// kModeBlockTail: the block product with the tail split of TcParams (an instantiation of its own, so that the kernel of the
+// large, multi-chunk products carries none of its geometry).
+enum Mode { kModeBlock = 0, kModeBlockTail = 1, kModeRowsum = 2, kModeRowsumSym = 3 };
 __host__ __device__ constexpr bool is_rowsum(int mode) { return mode == kModeRowsum || mode == kModeRowsumSym; }
 
 struct TcParams {
