@@ -47,7 +47,7 @@ struct Smem {
     static constexpr int kWHalf = is_rowsum(MODE) ? 0 : BT * 128;   // 64 j x BT columns fp16
     static constexpr int kWBytes = is_rowsum(MODE) ? 0 : 4 * kWHalf;   // [W_hi j-half 0][W_hi j-half 1][W_lo 0][W_lo 1]
     // symmetric row-sum mode: per-warp column partial sums, [row tile][parity][warp quarter][128 columns] floats
-    static constexpr int kColPartBytes = (MODE == kModeRowsumSym) ? 2 * 2 * 4 * 128 * 4 : 0;
+    static constexpr int kColPartBytes = (MODE == kModeRowsumSym) ? 2 * 2 * 4 * 128 * 4 + 64 : 0;   // + four mbarriers (col_ready[row tile][parity])
     static __host__ __device__ constexpr int stage_bytes(int K16) { return K16 * kXChunk + kWBytes; }
     static __host__ __device__ constexpr int total(int K16) {
         return 1024 /*align slack*/ + kStages * stage_bytes(K16) + 2 * K16 * kXChunk + 1024 /*barriers*/ + kColPartBytes;
@@ -68,10 +68,47 @@ struct Barriers {
     uint64_t p_half[kMaxBuf][2];            // block mode: first 64 columns of P written (lets the product MMA start early)
     uint64_t kw_done[kMaxBuf][2];           // block mode: product MMAs that read P from this buffer have completed
     uint64_t y_full[2], y_empty[2];         // accumulator flush hand-off (per row tile)
-    uint64_t col_ready[2][2];               // symmetric row-sum mode: the four warps' column partials of a tile are written
     uint32_t tmem_base;
     int abort_flag;
 };
+
+// ------------------------------------------------------------------------------------------------ work items
+// Work item w of a CTA -> (row pair, first column tile, number of column tiles, column chunk).
+//   block / row-sum modes: (column chunk c, row pair r) with c outermost, r = blockIdx.x + k * gridDim.x;
+//   block mode with tail split: full rounds first, then one half-range item of a tail pair (see TcParams);
+//   symmetric row-sum mode: only tiles on or above the diagonal.  Row pair r needs column tiles 2 r .. num_jt - 1; pairing r
+//     with num_work - 1 - r gives work units of equal length (num_jt + 2 tiles): unit u = blockIdx.x + k * gridDim.x is the
+//     two items {u, num_work - 1 - u} (the middle pair of an odd count stands alone: its second item is empty).
+struct ItemGeometry { int item, j0, num_jt, cch; bool tail_item; };
+
+template <int MODE>
+__device__ __forceinline__ ItemGeometry item_geometry(const TcParams& p, int w, int my_rows) {
+    ItemGeometry g;
+    if constexpr (MODE == kModeRowsumSym) {
+        const int unit = (int)blockIdx.x + (w >> 1) * (int)gridDim.x;
+        g.cch = 0;
+        g.item = (w & 1) ? p.num_work - 1 - unit : unit;
+        g.j0 = 2 * g.item;
+        g.num_jt = ((w & 1) && g.item == unit) ? 0 : p.num_jt - g.j0;
+        g.tail_item = false;
+    } else if constexpr (MODE == kModeBlockTail) {
+        const int full_rounds = p.tail_first / (int)gridDim.x;
+        const int half = (p.num_jt + 1) / 2;
+        g.cch = 0;
+        g.tail_item = w >= full_rounds;
+        const int part = g.tail_item ? (int)blockIdx.x / p.tail_pairs : 0;
+        g.item = g.tail_item ? p.tail_first + (int)blockIdx.x % p.tail_pairs : (int)blockIdx.x + w * (int)gridDim.x;
+        g.j0 = g.tail_item ? part * half : 0;
+        g.num_jt = g.tail_item ? (part == 0 ? half : p.num_jt - half) : p.num_jt;
+    } else {
+        g.cch = w / my_rows;
+        g.item = (int)blockIdx.x + (w % my_rows) * (int)gridDim.x;
+        g.j0 = g.cch * p.jt_chunk;
+        g.num_jt = (p.num_jt - g.j0 < p.jt_chunk) ? p.num_jt - g.j0 : p.jt_chunk;
+        g.tail_item = false;
+    }
+    return g;
+}
 
 // ------------------------------------------------------------------------------------------------ the kernel
 // Tiles of one work item are numbered n = 2 j + t (column tile j, row tile t) and flow through a ring of NBUF
@@ -105,8 +142,10 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 mbar_init(&bars->kw_done[u][t], 1); mbar_init(&bars->p_half[u][t], 4);
             }
         for (int t = 0; t < 2; ++t) { mbar_init(&bars->y_full[t], 1); mbar_init(&bars->y_empty[t], 4); }
-        for (int t = 0; t < 2; ++t)
-            for (int u = 0; u < 2; ++u) mbar_init(&bars->col_ready[t][u], 4);
+        if constexpr (MODE == kModeRowsumSym) {
+            uint64_t* col_ready = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(bars) + 1024 + 2 * 2 * 4 * 128 * 4);
+            for (int u = 0; u < 4; ++u) mbar_init(&col_ready[u], 4);          // the four warps' column partials of a tile are written
+        }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -123,33 +162,22 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
     // Work items of this CTA: (column chunk c, row-pair tile r) with c outermost, r = blockIdx.x + k * gridDim.x.  Every CTA
     // sweeps chunk c for all of its rows before chunk c + 1, so the whole grid reads the same L2-sized slice of the
     // column operands at about the same time; a row's partial results always come from the same threads, in order.
-    //
-    // Symmetric row-sum mode: only tiles on or above the diagonal are evaluated.  Row pair r needs column tiles 2 r .. num_jt - 1;
-    // pairing r with num_work - 1 - r gives every CTA work units of equal length (num_jt + 2 tiles): unit u = blockIdx.x +
-    // k * gridDim.x is the two items {u, num_work - 1 - u} (the middle pair of an odd count stands alone: its second
-    // item is empty).
+    // (item_geometry above has the other modes' orders.)
     constexpr bool kSym = MODE == kModeRowsumSym;
-    const int sym_units = (p.num_work + 1) / 2;
     constexpr bool kTail = MODE == kModeBlockTail;
-    const int full_rounds = kTail ? p.tail_first / (int)gridDim.x : 0;
-    const int my_rows = kSym ? (sym_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
+    const int my_rows = kSym ? ((p.num_work + 1) / 2 - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
                              : (p.num_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int my_items = kSym ? 2 * my_rows
-                       : kTail ? full_rounds + ((int)blockIdx.x < 2 * p.tail_pairs ? 1 : 0) : my_rows * p.num_chunks;
-    const int tail_half = (p.num_jt + 1) / 2;
+                       : kTail ? p.tail_first / (int)gridDim.x + ((int)blockIdx.x < 2 * p.tail_pairs ? 1 : 0) : my_rows * p.num_chunks;
 #define FD_ITEM_GEOMETRY(w)                                                                         \
-    const bool tail_item = kTail && (w) >= full_rounds;                                             \
-    const int tail_part = tail_item ? (int)blockIdx.x / p.tail_pairs : 0;                           \
-    const int unit_ = (int)blockIdx.x + (kSym ? ((w) >> 1) : kTail ? (w) : ((w) % my_rows)) * (int)gridDim.x;     \
-    const int cch = (kSym || kTail) ? 0 : (w) / my_rows;                                            \
-    const int item = tail_item ? p.tail_first + (int)blockIdx.x % p.tail_pairs                      \
-                               : (kSym && ((w) & 1)) ? p.num_work - 1 - unit_ : unit_;              \
-    const int j0 = kSym ? 2 * item : tail_item ? tail_part * tail_half : cch * p.jt_chunk;          \
-    const int num_jt = kSym ? ((((w) & 1) && item == unit_) ? 0 : p.num_jt - j0)                    \
-                     : tail_item ? (tail_part == 0 ? tail_half : p.num_jt - tail_half)              \
-                            : ((p.num_jt - j0 < p.jt_chunk) ? p.num_jt - j0 : p.jt_chunk);          \
+    const ItemGeometry geo_ = item_geometry<MODE>(p, (w), my_rows);                                 \
+    const int cch = geo_.cch;                                                                       \
+    const int item = geo_.item;                                                                     \
+    const int j0 = geo_.j0;                                                                         \
+    const int num_jt = geo_.num_jt;                                                                 \
+    const bool tail_item = geo_.tail_item;                                                          \
     const int tiles_per_item = 2 * num_jt;                                                          \
-    (void)tail_item; (void)tail_part;                                                               \
+    (void)tail_item;                                                                                \
     (void)item; (void)tiles_per_item; (void)cch
     const int flush = p.flush;
 
@@ -405,6 +433,7 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                 constexpr int kSymFlush = 64;
                 constexpr bool kWantSq = BT == 16;             // the sum of squares rides along in the first degree pass only (BT = 32: without)
                 float* colpart = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 1024);
+                uint64_t* col_ready = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(bars) + 1024 + 2 * 2 * 4 * 128 * 4);
                 const double fix = (double)(1ull << p.sym_shift);
                 const int It = 2 * item + t;
                 float acc[128];
@@ -433,8 +462,8 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
 #pragma unroll
                     for (int c = 0; c < 128; ++c) acc[c] = 0.f;
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->col_ready[t][slot]);
-                    if (!mbar_wait(&bars->col_ready[t][slot], (ncol >> 1) & 1u, abort_flag, p.status, 11)) return false;
+                    if (lane == 0) mbar_arrive(&col_ready[t * 2 + slot]);
+                    if (!mbar_wait(&col_ready[t * 2 + slot], (ncol >> 1) & 1u, abort_flag, p.status, 11)) return false;
                     const float* all = colpart + ((t * 2 + (int)slot) * 4) * 128;
                     const int cidx = wq * 32 + lane;
                     const float csum = (all[cidx] + all[128 + cidx]) + (all[256 + cidx] + all[384 + cidx]);
