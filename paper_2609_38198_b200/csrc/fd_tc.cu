@@ -906,7 +906,7 @@ fd_status apply_tc(fd_ctx* c, const ApplyArgs& a) {
         const int sym_grid = std::min((p.num_work + 1) / 2, c->sm_count);
         if (p.rowsq) FD_TRY((launch_tc<16, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
         else FD_TRY((launch_tc<32, kModeRowsumSym>(c, mr, mc, mc, mc, p, sym_grid)));
-        k_sym_finish<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(p.symsum, N, std::ldexp(1.0, -(kBias + p.sym_shift)), a.Y);
+        k_sym_finish<<<(unsigned)ceil_div(N, 256), 256, 0, c->stream>>>(p.symsum, N, std::ldexp(1.0, -(kBias + (int)p.sym_shift)), a.Y);
         FD_LAUNCH_CHECK(c, "k_sym_finish");
     } else if (rowsum) {
         p.q = a.Y; p.rowsq = a.rowsq; p.b = 1;

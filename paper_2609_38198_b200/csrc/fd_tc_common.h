@@ -26,12 +26,6 @@ struct TcParams {
     int num_work;                // row-pair tiles (256 rows each)
     int num_jt;                  // column tiles
     int jt_chunk, num_chunks;    // the column range is swept in chunks small enough for L2 (block mode); all CTAs work on one chunk at a time
-    // Tail split (block mode with a single column chunk): the row pairs left over after the full rounds -- all of them when
-    // there are fewer pairs than CTAs -- are each served by TWO CTAs, one per half of the column range, whose partial
-    // results meet in Y by atomic addition (Y zeroed beforehand; a sum of two terms does not depend on their order).
-    int tail_split;              // 0 = off, 2 = on
-    int tail_first;              // first row pair of the tail
-    int tail_pairs;              // number of row pairs in the tail
     int64_t np_rows;             // padded row count of the operand arrays (row index of K slab c = c * np + p)
     int64_t np_cols;
     int K16;
@@ -39,12 +33,27 @@ struct TcParams {
     int flush;                   // column tiles per accumulator flush
     const float* left;           // may be null
     const float* colscale_inv;   // per column: 2^-bias / colscale
-    float* Y; int64_t ldy;
-    float* q; double* rowsq;     // row-sum outputs
-    unsigned long long* symsum;  // symmetric row-sum mode: fixed-point row + column sums, one 64-bit integer per point
-    int sym_shift;               // ... in units of 2^-sym_shift of the (2^bias-scaled) kernel values
+    // The parameter block keeps the size it had with the block and row-sum outputs alone (the block product's kernel
+    // measured 2.5 % more SM cycles with a larger one): the modes added later borrow the fields their mode does not use.
+    union {
+        struct { float* Y; int64_t ldy; };                       // block modes: output block
+        struct { unsigned long long* symsum; int64_t sym_shift; };   // symmetric row-sum mode: fixed-point row + column sums, one
+                                                                 // 64-bit integer per point, in units of 2^-sym_shift of the
+                                                                 // (2^bias-scaled) kernel values
+    };
+    union {
+        struct { float* q; double* rowsq; };                     // row-sum modes: outputs
+        // Tail split (block mode with a single column chunk): the row pairs left over after the full rounds -- all of them
+        // when there are fewer pairs than CTAs -- are each served by TWO CTAs, one per half of the column range, whose
+        // partial results meet in Y by atomic addition (Y zeroed beforehand; a sum of two terms does not depend on order).
+        struct { int tail_split;                                 // 0 = off, 2 = on
+                 int tail_first;                                 // first row pair of the tail
+                 int tail_pairs;                                 // number of row pairs in the tail
+                 int tail_pad_; };
+    };
     unsigned int* status;
 };
+static_assert(sizeof(TcParams) == 120, "the kernels' parameter block has a measured size");
 
 // ------------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
