@@ -31,6 +31,7 @@ struct TcParams {
     int K16;
     int b;                       // real block columns to store
     int flush;                   // column tiles per accumulator flush
+    int lo_row;                  // block modes: first row of W_lo inside the W operand array (W_hi starts at row 0)
     const float* left;           // may be null
     const float* colscale_inv;   // per column: 2^-bias / colscale
     // The parameter block keeps the size it had with the block and row-sum outputs alone (the block product's kernel
