@@ -645,7 +645,10 @@ k_tc(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                             float* o = p.Y + row + (int64_t)c * p.ldy;
                             const float v = acc[c] * l * p.colscale_inv[c];
                             if (kTail && tail_item) atomicAdd(o, v);   // the other half of the column range arrives from another CTA
-                            else *o = cch == 0 ? v : *o + v;           // later column chunks add to the partial result of the same thread
+                            // later column chunks add to the partial result of the same thread; streaming loads and stores:
+                            // the partial results are touched once per chunk round and should not push the fp16 operands,
+                            // which every CTA re-reads, out of L2
+                            else __stcs(o, cch == 0 ? v : __ldcs(o) + v);
                         }
                 }
             }

@@ -300,7 +300,7 @@ k_bp(const __grid_constant__ CUtensorMap map_xrow, const __grid_constant__ CUten
                     if (c < p.b) {
                         float* o = p.Y + row + (int64_t)c * p.ldy;
                         const float v = acc[c] * l * p.colscale_inv[c];
-                        *o = cch == 0 ? v : *o + v;          // later column chunks add to the partial result of the same thread
+                        __stcs(o, cch == 0 ? v : __ldcs(o) + v);   // later column chunks add to the partial result of the same thread (streaming: touched once per chunk round)
                     }
             }
         }
