@@ -86,7 +86,8 @@ fd_status fd_create(fd_ctx** out, const float* X_dev, int64_t N, int32_t D, int6
 fd_status fd_destroy(fd_ctx* ctx);
 
 /* Tuning / test knobs by name: "path" (FD_PATH_*), "splits" (0 = auto), "flush" (column tiles
- * between accumulator flushes of the tensor-core kernel), "tc_max_mag" (largest beta * log2(e) *
+ * between accumulator flushes of the tensor-core kernels; 0 = default: 1 in the fp32-grade mode, whose eigenvalue budget
+ * the tensor core's round-toward-zero accumulation would otherwise eat, 8 in the reduced-precision mode), "tc_max_mag" (largest beta * log2(e) *
  * max|x - mu|^2 for which the Gram-form tensor-core kernel serves the fp32 mode), "jt_chunk" (column
  * tiles per L2-resident chunk of the tensor-core block product), "sym" (1, default: the degree passes on the Gram-form
  * kernels use K = K^T and evaluate only the tiles on or above the diagonal -- each off-diagonal tile gives the row sums
