@@ -232,3 +232,23 @@ def test_torch_distributed_transport_on_a_one_rank_group(fd, dev):
         ctx.close()
     finally:
         dist.destroy_process_group()
+
+
+def test_eigs_sharded_with_a_rank_that_owns_no_rows(fd, dev):
+    # 500 points on 3 ranks: ranges (0, 256), (256, 500), (500, 500) -- the last rank owns nothing, contributes zeros to every
+    # sum and still has to take every decision the others take
+    N, beta, alpha, k, b = 500, 0.4, 1.0, 6, 8
+    X = workloads.torus6(N, seed=12)
+    lam_o, U_o, d_o = dense.eigs(X, beta, alpha, k)
+    assert fd.fd_shard_rows(N, 3, 2) == (500, 500)
+
+    def body(ctx, r):
+        ctx.degree(beta, alpha)
+        lam, U, info = ctx.eigs(k, b)
+        return lam, U.cpu().numpy(), info.converged
+
+    res = run_ranks(fd, dev, 3, X, b, 64, body)
+    for r in range(3):
+        lam, U, conv = res[r]
+        assert conv == k + 1 and np.abs(lam - lam_o).max() <= 1e-6
+        assert np.array_equal(lam, res[0][0]) and np.array_equal(U, res[0][1])
