@@ -24,8 +24,7 @@ a lattice torus; two-point and simplex closed forms; K(2 beta) = K(beta)^2; n_ef
 k equal weights; dense eigh vs the blocked path; Nystrom reproduces psi at sample points;
 principal angles and the RV score on subspaces with known angles; the cascade on a
 hand-built potential.  The beta-flow's bracket rule and the cascade's hand-over rule have
-only soft pins against the paper (its printed T^6 table, another RNG; for N >= 2^17, where
-the paper prints single runs, the GPU flow reproduces the printed bandwidths to three
-digits): exact beta-flow parity is "parity unpinned".
+only soft pins against the paper (its printed T^6 table, another RNG): exact beta-flow
+parity is "parity unpinned".
 """
 from . import dense, blocked, flow, nystrom, overlap  # noqa: F401
