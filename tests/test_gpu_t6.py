@@ -89,3 +89,15 @@ def test_sweep_follows_the_printed_table(fd, dev):
     assert all(b1 > b0 for b0, b1 in zip(bxs[:6], bxs[1:7]))
     # trend: the first-harmonic error falls by more than an order of magnitude from 2^10 to 2^17
     assert (1.0 - res[1 << 17][1]) < 0.1 * (1.0 - res[1024][1])
+
+
+@pytest.mark.parametrize("log2n", [18, 19])
+def test_larger_sizes_match_the_printed_single_runs(fd, dev, log2n):
+    """N = 2^18 and 2^19: the paper prints one run each (seed 42, another RNG); the selected bandwidth must match to 1 % and the
+    first-harmonic error to 30 % (measured: 0.2 % / 0.03 % and 11 % / 12 %)."""
+    N = 1 << log2n
+    tab = table()
+    X, ang, bx, status, lam, psi, recs, score, path = gpu_run(fd, dev, N, 42)
+    assert status == "VERTEX" and path == fd.FD_PATH_TC
+    assert abs(bx / tab[N][0] - 1.0) < 0.01, (bx, tab[N][0])
+    assert abs((1.0 - score) / (1.0 - tab[N][2]) - 1.0) < 0.3, (1.0 - score, 1.0 - tab[N][2])
